@@ -1,0 +1,245 @@
+/*
+ * relaxkv.h - C ABI of the RelaxKV selective cache-repair hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, the two halves of the repair path of
+ * "RelaxKV: Recomputation Guided by the Query with Sparse Context Attention":
+ *   (a) query-guided anchor selection   - relaxkv_score_select, relaxkv_build_active_sets
+ *   (b) sparse-context repair attention - relaxkv_sparse_ctx_attention, relaxkv_scatter_kv
+ *
+ * General conventions (they hold for every entry point unless it says otherwise)
+ * -----------------------------------------------------------------------------
+ * Pointers.   A name starting with h_ is a HOST pointer, read during the call only.  Every other
+ *             pointer is a DEVICE pointer of the current CUDA device.  All buffers are owned by the
+ *             caller; the library allocates nothing, frees nothing and keeps no pointer after the
+ *             call returns.  Scratch comes from the caller's `workspace` (device memory, 256-byte
+ *             aligned, at least relaxkv_workspace_bytes() bytes).
+ * Types.      K, V, Q and attention outputs are bf16 (2 bytes); scores are fp32; every index is
+ *             int32.  head_dim is contiguous in memory everywhere.  bf16 base pointers must be
+ *             16-byte aligned and the cache strides multiples of 8 elements.
+ * Batching.   A call covers n_req independent requests (a ragged batch).  Per-request arrays are
+ *             packed back to back; "cu" arrays hold the n_req+1 exclusive prefix offsets.
+ * Positions.  Context positions are request-local token indices 0..T_c-1.  Every index list is
+ *             ascending and free of duplicates.  Active targets are stored as ranks into the
+ *             sorted union U, so a target's causal limit is its own rank.
+ * Heads.      Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ * Asynchrony. All work is enqueued on `stream`; no call synchronises except
+ *             relaxkv_read_device_status.  Data-dependent set sizes stay on the device; the host
+ *             passes upper bounds.
+ * Errors.     Host-checkable violations (NULL, bad shape, misalignment, workspace too small) return
+ *             a status before any launch.  Launch failures return RELAXKV_ERR_CUDA.  Problems only
+ *             the device can see (an index out of range, a count above its host bound, a bounded
+ *             wait that expired) are recorded in a device status word - the kernel skips the
+ *             offending work and returns normally - and are read with relaxkv_read_device_status.
+ * Precision.  bf16 inputs, fp32 accumulation and softmax, probabilities rounded to bf16 before the
+ *             P*V product, bf16 outputs.
+ */
+#ifndef RELAXKV_H_
+#define RELAXKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RELAXKV_OK = 0,
+  RELAXKV_ERR_INVALID_ARG = 1,
+  RELAXKV_ERR_UNSUPPORTED_SHAPE = 2,
+  RELAXKV_ERR_WORKSPACE_TOO_SMALL = 3,
+  RELAXKV_ERR_CUDA = 4,
+  RELAXKV_ERR_BAD_INDEX = 5,
+  RELAXKV_ERR_TIMEOUT = 6
+} relaxkv_status;
+
+/* A CUDA stream handle (cudaStream_t) passed as an opaque pointer; NULL is the default stream. */
+typedef void* relaxkv_stream;
+
+/* Shapes shared by all calls. */
+typedef struct {
+  int32_t n_req;              /* 1 <= B <= 64 requests in the batch                             */
+  int32_t n_q_heads;          /* H                                                              */
+  int32_t n_kv_heads;         /* H_kv, divides H; the group size G = H / H_kv must be <= 16     */
+  int32_t head_dim;           /* D, 64 or 128                                                   */
+  const int32_t* h_ctx_len;   /* host [B]: context tokens T_c of each request                   */
+  const int32_t* h_q_len;     /* host [B]: query-suffix tokens Q of each request; read by       */
+                              /* relaxkv_score_select and relaxkv_workspace_bytes only          */
+  float softmax_scale;        /* multiplies q.k before the softmax (usually 1/sqrt(D))          */
+} relaxkv_shape;
+
+/* One layer's KV cache.  Element (request b, token i, kv head g, dim d) of K lives at
+ * k + (h_req_token_offset[b] + i) * token_stride + g * head_stride + d  (in elements), same for V.
+ * This covers [tokens, H_kv, D] and [H_kv, tokens, D] storage. */
+typedef struct {
+  void* k;
+  void* v;
+  int64_t token_stride;
+  int64_t head_stride;
+  const int64_t* h_req_token_offset;   /* host [B]: first token row of each request */
+} relaxkv_cache_view;
+
+/* How the recomputation context of a target at position p is built. */
+typedef enum {
+  RELAXKV_CTX_UNION = 0,        /* C_l(p) = U intersect {j <= p}  (the method)                    */
+  RELAXKV_CTX_FULL_PREFIX = 1   /* every position j <= p (the paper's Full-Prefix Control)        */
+} relaxkv_ctx_mode;
+
+const char* relaxkv_status_string(int32_t status);
+
+/* Anchors per layer, k = max(1, round(r * T_c)) clamped to T_c; round is to nearest with halves to
+ * even on the fp64 product.  (Appendix A.1, anchor-count equation; Section 3.2.)  Host only. */
+int32_t relaxkv_anchor_count(int32_t ctx_len, double ratio);
+
+/* Bytes of device scratch that suffice for any call below with these shapes.  h_k may be NULL.
+ * Returns 0 for an invalid shape.  Host only. */
+size_t relaxkv_workspace_bytes(const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k);
+
+/*
+ * Query-attention scoring and per-layer top-k anchors (Section 3.2, score equation and TopK;
+ * Algorithm 1, steps 1-5; Appendix A.1).
+ *
+ * For each layer l < n_layers and request b, with Q = the request's query-suffix rows:
+ *   s[h,t,i]  = softmax_scale * <q[t,h,:], K[i, h/G, :]>                i over all T_c cached tokens
+ *   A[h,t,i]  = exp(s[h,t,i] - lse[h,t])     lse = log sum_i exp(s[h,t,i])  unless supplied
+ *   raw[i]    = (1/(H*Q)) * sum_h sum_t A[h,t,i]
+ *   norm[i]   = (raw[i] - min raw) / (max raw - min raw)                (all zeros if max == min)
+ *   anchors   = positions of the k largest raw[i]; equal scores go to the lower position;
+ *               written in ascending order.  (MinMax is monotone, so selecting on raw selects the
+ *               same set as selecting on norm.)
+ *
+ * q_layers         host array [n_layers] of device bf16 [sum_b Q_b, H, D] (requests packed).
+ * cache_layers     host array [n_layers]; only .k is read.
+ * row_lse_layers   NULL, or host array [n_layers] of device fp32 [H, sum_b Q_b] (entry (h, row));
+ *                  when given for a layer, its rows' log-normalisers are taken from it (e.g. from the
+ *                  query's own forward pass, whose softmax also spans the query tokens) and the
+ *                  statistics pass is skipped.  An entry may itself be NULL.
+ * h_k              host [B]: anchors per layer for each request, 1 <= k_b <= T_c.
+ * raw_scores_out   device fp32 [n_layers, sum_b T_c].
+ * norm_scores_out  NULL or device fp32 [n_layers, sum_b T_c].
+ * anchors_out      device int32 [n_layers, sum_b k_b]; request-local positions.
+ * Results are deterministic: reductions run in a fixed order (no floating-point atomics).
+ */
+relaxkv_status relaxkv_score_select(
+    const relaxkv_shape* shape, int32_t n_layers,
+    const void* const* q_layers, const relaxkv_cache_view* cache_layers,
+    const float* const* row_lse_layers, const int32_t* h_k,
+    float* raw_scores_out, float* norm_scores_out, int32_t* anchors_out,
+    void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/*
+ * The selection step of relaxkv_score_select on its own (Appendix A.1, TopK; Section 3.2, MinMax):
+ * top-k anchors (and optionally the MinMax-normalised scores) of given raw scores.  Same layouts,
+ * tie rule and output order as above.  Exists so the step can be checked and timed by itself.
+ */
+relaxkv_status relaxkv_select_topk(
+    const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const float* raw_scores,
+    float* norm_scores_out, int32_t* anchors_out, relaxkv_stream stream);
+
+/*
+ * Repair schedule from the per-layer anchors (Section 3.2, definitions of h_i, U, R_l;
+ * Algorithm 1, steps 6-12; Appendix A.2, "stored in sorted order and mapped to compact indices").
+ *
+ *   h_i  = max{ l : i in S_l }  (-1 if i is in no S_l);   U = { i : h_i >= 0 } ascending;
+ *   u_rank[i] = index of i in U (or -1);   R_l = { c : h_{U[c]} >= l } as ascending ranks c.
+ *
+ * anchors            device int32 [n_layers, sum_b k_b] as written by relaxkv_score_select.
+ * highest_layer_out  device int32 [sum_b T_c].
+ * u_pos_out          device int32, capacity sum_b min(T_c, n_layers*k_b): U of each request, packed.
+ * u_cu_out           device int32 [B+1].
+ * u_rank_out         device int32 [sum_b T_c].
+ * r_rank_out         device int32, capacity n_layers * (capacity of u_pos_out): for layer l and
+ *                    request b the ranks of R_{l,b}, packed in (l, b) order.
+ * r_cu_out           device int32 [n_layers*B + 1]: offset of segment (l, b) at index l*B + b.
+ * h_counts_pinned    NULL or pinned host int32 [B + n_layers*B]: |U_b| then |R_{l,b}|; valid once
+ *                    the stream has been synchronised.
+ */
+relaxkv_status relaxkv_build_active_sets(
+    const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
+    int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
+    int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned,
+    void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/*
+ * Sparse-context repair attention of one layer (Section 3.3, C_l(p); Section 3.4, mixed
+ * fresh/cached K/V; Algorithm 1, steps 16-19; Appendix A.2).
+ *
+ * Target row rho of request b has rank c* = r_rank[r_cu_layer[b] + rho] in U_b and position
+ * p = u_pos[u_cu[b] + c*].  With the context list X = U_b (RELAXKV_CTX_UNION; limit = c*) or
+ * X = (0..T_c-1) (RELAXKV_CTX_FULL_PREFIX; limit = p), and
+ *   Kt[x] = k_new[row of x] if X[x] is an active target of this layer, else cache K at X[x]
+ * (same for V), the call computes for every query head h
+ *   out[rho,h,:] = sum_{x <= limit} softmax_x(softmax_scale * <q_new[rho,h,:], Kt[x, h/G, :]>) * Vt[x, h/G, :]
+ * The target itself is part of its context.  The cache is not modified.
+ *
+ * q_new           device bf16 [n_target_rows, H, D]; the rows of request b start at
+ *                 r_cu_layer[b] - r_cu_layer[0] and follow the order of its R list.
+ * k_new, v_new    device bf16 [n_target_rows, H_kv, D], or both NULL to read the cache only.
+ * u_pos, u_cu     as written by relaxkv_build_active_sets.
+ * r_rank          base of the packed rank array written by relaxkv_build_active_sets.
+ * r_cu_layer      r_cu_out + l*B for this layer (B+1 offsets into r_rank are read).
+ * n_target_rows   rows allocated in q_new/k_new/v_new/out (>= the layer's true total).
+ * h_max_targets   host [B]: upper bound of |R_{l,b}|.   h_max_ctx: host [B]: upper bound of |U_b|.
+ *                 A true count above its bound is reported through the device status word.
+ * out             device bf16 [n_target_rows, H, D].
+ * lse_out         NULL or device fp32 [H, n_target_rows]: log-normaliser of each output row.
+ */
+relaxkv_status relaxkv_sparse_ctx_attention(
+    const relaxkv_shape* shape, relaxkv_ctx_mode mode, const relaxkv_cache_view* cache,
+    const void* q_new, const void* k_new, const void* v_new,
+    const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
+    int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
+    void* out, float* lse_out,
+    void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/*
+ * Cache update of one layer (Section 3.4; Algorithm 1, step 21): the fresh K/V of every active
+ * target overwrite its cache entry; no other byte of the cache changes.  Idempotent.
+ * Arguments as for relaxkv_sparse_ctx_attention; `cache` is written in place.
+ */
+relaxkv_status relaxkv_scatter_kv(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache,
+    const void* k_new, const void* v_new,
+    const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
+    const int32_t* h_max_targets, relaxkv_stream stream);
+
+/*
+ * Materialised mixed context of one layer (Section 3.4 equation; Algorithm 1, steps 17-18):
+ * k_ctx_out / v_ctx_out, device bf16 [ctx_rows, H_kv, D], receive for request b, at rows
+ * x_cu[b] .. , Kt/Vt of the context list X defined above, where x_cu = u_cu (UNION) or the prefix
+ * sums of T_c (FULL_PREFIX).  The 128 rows after the last one are zero-filled (as far as ctx_rows
+ * allows).  ctx_rows >= sum_b h_max_ctx[b] (UNION) or sum_b T_c (FULL_PREFIX).
+ * relaxkv_sparse_ctx_attention runs this step itself into its workspace; the entry point exists
+ * so the step can be checked and timed on its own.
+ */
+relaxkv_status relaxkv_gather_kv(
+    const relaxkv_shape* shape, relaxkv_ctx_mode mode, const relaxkv_cache_view* cache,
+    const void* k_new, const void* v_new,
+    const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
+    const int32_t* h_max_ctx, void* k_ctx_out, void* v_ctx_out, int64_t ctx_rows,
+    relaxkv_stream stream);
+
+/*
+ * Test utility: the same result as relaxkv_sparse_ctx_attention from a plain SIMT kernel (one warp
+ * per output row, fp32 throughout, no tensor cores).  A second opinion for debugging; far slower.
+ */
+relaxkv_status relaxkv_sparse_ctx_attention_simt(
+    const relaxkv_shape* shape, relaxkv_ctx_mode mode, const relaxkv_cache_view* cache,
+    const void* q_new, const void* k_new, const void* v_new,
+    const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
+    int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
+    void* out, float* lse_out,
+    void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/*
+ * Synchronises `stream`, copies the device status word (a relaxkv_status: RELAXKV_OK,
+ * RELAXKV_ERR_BAD_INDEX or RELAXKV_ERR_TIMEOUT, the first problem recorded wins) to
+ * *h_status_out and clears it.  h_detail_out (NULL or host int32[4]) receives where it happened:
+ * kernel id, block, and two kernel-specific values.
+ */
+relaxkv_status relaxkv_read_device_status(int32_t* h_status_out, int32_t* h_detail_out, relaxkv_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* RELAXKV_H_ */

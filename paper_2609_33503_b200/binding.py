@@ -1,0 +1,232 @@
+"""Python binding of the RelaxKV C ABI (include/relaxkv.h): argument marshalling only.
+
+Every function here has the name of the C entry point it calls and does nothing but turn torch
+tensors and Python lists into pointers and sizes.  All computation runs in the CUDA kernels of
+librelaxkv.so; there is no CPU path and no fallback: if the library has not been built, loading
+fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librelaxkv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_INDEX, ERR_TIMEOUT = range(7)
+CTX_UNION, CTX_FULL_PREFIX = 0, 1
+
+ENTRY_POINTS = (
+    "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
+    "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
+    "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
+)
+
+
+class RelaxKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("n_req", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("h_ctx_len", ctypes.POINTER(ctypes.c_int32)),
+                ("h_q_len", ctypes.POINTER(ctypes.c_int32)), ("softmax_scale", ctypes.c_float)]
+
+
+class _CacheView(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("token_stride", ctypes.c_int64),
+                ("head_stride", ctypes.c_int64), ("h_req_token_offset", ctypes.POINTER(ctypes.c_int64))]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_33503_b200.build` "
+                               "(nvcc, sm_100a). There is no CPU fallback.")
+        l = ctypes.CDLL(LIB_PATH)
+        l.relaxkv_status_string.restype = ctypes.c_char_p
+        l.relaxkv_status_string.argtypes = [ctypes.c_int32]
+        l.relaxkv_anchor_count.restype = ctypes.c_int32
+        l.relaxkv_anchor_count.argtypes = [ctypes.c_int32, ctypes.c_double]
+        l.relaxkv_workspace_bytes.restype = ctypes.c_size_t
+        l.relaxkv_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
+        for name in ENTRY_POINTS[3:]:
+            getattr(l, name).restype = ctypes.c_int32
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().relaxkv_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise RelaxKVError(status, where)
+
+
+def _i32(xs: Optional[Sequence[int]]):
+    if xs is None:
+        return None
+    return (ctypes.c_int32 * len(xs))(*[int(x) for x in xs])
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(None) if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+class Shape:
+    """Host-side relaxkv_shape; keeps its arrays alive."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, ctx_lens: Sequence[int],
+                 q_lens: Optional[Sequence[int]] = None, softmax_scale: Optional[float] = None):
+        self.ctx_lens = [int(x) for x in ctx_lens]
+        self.q_lens = None if q_lens is None else [int(x) for x in q_lens]
+        self._ctx = _i32(self.ctx_lens)
+        self._q = _i32(self.q_lens)
+        self.c = _Shape()
+        self.c.n_req = len(self.ctx_lens)
+        self.c.n_q_heads, self.c.n_kv_heads, self.c.head_dim = int(n_q_heads), int(n_kv_heads), int(head_dim)
+        self.c.h_ctx_len = ctypes.cast(self._ctx, ctypes.POINTER(ctypes.c_int32))
+        self.c.h_q_len = ctypes.cast(self._q, ctypes.POINTER(ctypes.c_int32)) if self._q is not None else None
+        self.c.softmax_scale = float(softmax_scale if softmax_scale is not None else head_dim ** -0.5)
+
+    @property
+    def n_req(self) -> int:
+        return len(self.ctx_lens)
+
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+class CacheView:
+    """Host-side relaxkv_cache_view over torch tensors k, v of logical shape [tokens, H_kv, D]
+    (any token/head strides, D contiguous); requests start at the given token rows."""
+
+    def __init__(self, k: torch.Tensor, v: Optional[torch.Tensor], req_token_offsets: Sequence[int]):
+        assert k.dim() == 3 and k.stride(2) == 1 and k.dtype == torch.bfloat16
+        if v is not None:
+            assert v.shape == k.shape and v.stride() == k.stride() and v.dtype == torch.bfloat16
+        self.k, self.v = k, v
+        self._off = (ctypes.c_int64 * len(req_token_offsets))(*[int(x) for x in req_token_offsets])
+        self.c = _CacheView()
+        self.c.k = k.data_ptr()
+        self.c.v = v.data_ptr() if v is not None else None
+        self.c.token_stride, self.c.head_stride = int(k.stride(0)), int(k.stride(1))
+        self.c.h_req_token_offset = ctypes.cast(self._off, ctypes.POINTER(ctypes.c_int64))
+
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def relaxkv_anchor_count(ctx_len: int, ratio: float) -> int:
+    return int(lib().relaxkv_anchor_count(int(ctx_len), float(ratio)))
+
+
+def relaxkv_workspace_bytes(shape: Shape, n_layers: int, k: Optional[Sequence[int]] = None) -> int:
+    return int(lib().relaxkv_workspace_bytes(shape.ref(), int(n_layers), _i32(k)))
+
+
+def relaxkv_score_select(shape: Shape, q_layers: List[torch.Tensor], cache_layers: List[CacheView],
+                         k: Sequence[int], raw_scores_out: torch.Tensor, anchors_out: torch.Tensor,
+                         workspace: torch.Tensor, norm_scores_out: Optional[torch.Tensor] = None,
+                         row_lse_layers: Optional[List[Optional[torch.Tensor]]] = None, stream=None) -> None:
+    n_layers = len(q_layers)
+    qs = (ctypes.c_void_p * n_layers)(*[q.data_ptr() for q in q_layers])
+    caches = (_CacheView * n_layers)(*[c.c for c in cache_layers])
+    lses = None
+    if row_lse_layers is not None:
+        lses = (ctypes.c_void_p * n_layers)(*[(t.data_ptr() if t is not None else None) for t in row_lse_layers])
+    _check(lib().relaxkv_score_select(shape.ref(), n_layers, qs, caches, lses, _i32(k), _ptr(raw_scores_out),
+                                      _ptr(norm_scores_out), _ptr(anchors_out), _ptr(workspace),
+                                      ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)),
+           "relaxkv_score_select")
+
+
+def relaxkv_select_topk(shape: Shape, n_layers: int, k: Sequence[int], raw_scores: torch.Tensor,
+                        anchors_out: torch.Tensor, norm_scores_out: Optional[torch.Tensor] = None,
+                        stream=None) -> None:
+    _check(lib().relaxkv_select_topk(shape.ref(), int(n_layers), _i32(k), _ptr(raw_scores), _ptr(norm_scores_out),
+                                     _ptr(anchors_out), _stream(stream)), "relaxkv_select_topk")
+
+
+def relaxkv_build_active_sets(shape: Shape, n_layers: int, k: Sequence[int], anchors: torch.Tensor,
+                              highest_layer_out: torch.Tensor, u_pos_out: torch.Tensor, u_cu_out: torch.Tensor,
+                              u_rank_out: torch.Tensor, r_rank_out: torch.Tensor, r_cu_out: torch.Tensor,
+                              workspace: torch.Tensor, counts_pinned: Optional[torch.Tensor] = None,
+                              stream=None) -> None:
+    _check(lib().relaxkv_build_active_sets(shape.ref(), int(n_layers), _i32(k), _ptr(anchors),
+                                           _ptr(highest_layer_out), _ptr(u_pos_out), _ptr(u_cu_out),
+                                           _ptr(u_rank_out), _ptr(r_rank_out), _ptr(r_cu_out), _ptr(counts_pinned),
+                                           _ptr(workspace),
+                                           ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                           _stream(stream)),
+           "relaxkv_build_active_sets")
+
+
+def _attention(fn_name, shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, max_targets,
+               max_ctx, out, lse_out, workspace, stream):
+    fn = getattr(lib(), fn_name)
+    _check(fn(shape.ref(), int(mode), cache.ref(), _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(u_pos), _ptr(u_cu),
+              _ptr(r_rank), _ptr(r_cu_layer), ctypes.c_int64(q_new.shape[0]), _i32(max_targets), _i32(max_ctx),
+              _ptr(out), _ptr(lse_out), _ptr(workspace),
+              ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)), fn_name)
+
+
+def relaxkv_sparse_ctx_attention(shape: Shape, mode: int, cache: CacheView, q_new: torch.Tensor,
+                                 k_new: Optional[torch.Tensor], v_new: Optional[torch.Tensor],
+                                 u_pos: torch.Tensor, u_cu: torch.Tensor, r_rank: torch.Tensor,
+                                 r_cu_layer: torch.Tensor, max_targets: Sequence[int], max_ctx: Sequence[int],
+                                 out: torch.Tensor, workspace: torch.Tensor,
+                                 lse_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """n_target_rows is q_new.shape[0]; k_new/v_new/out must have as many rows."""
+    _attention("relaxkv_sparse_ctx_attention", shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank,
+               r_cu_layer, max_targets, max_ctx, out, lse_out, workspace, stream)
+
+
+def relaxkv_sparse_ctx_attention_simt(shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer,
+                                      max_targets, max_ctx, out, workspace, lse_out=None, stream=None) -> None:
+    _attention("relaxkv_sparse_ctx_attention_simt", shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank,
+               r_cu_layer, max_targets, max_ctx, out, lse_out, workspace, stream)
+
+
+def relaxkv_scatter_kv(shape: Shape, cache: CacheView, k_new: torch.Tensor, v_new: torch.Tensor,
+                       u_pos: torch.Tensor, u_cu: torch.Tensor, r_rank: torch.Tensor, r_cu_layer: torch.Tensor,
+                       max_targets: Sequence[int], stream=None) -> None:
+    _check(lib().relaxkv_scatter_kv(shape.ref(), cache.ref(), _ptr(k_new), _ptr(v_new), _ptr(u_pos), _ptr(u_cu),
+                                    _ptr(r_rank), _ptr(r_cu_layer), _i32(max_targets), _stream(stream)),
+           "relaxkv_scatter_kv")
+
+
+def relaxkv_gather_kv(shape: Shape, mode: int, cache: CacheView, k_new: Optional[torch.Tensor],
+                      v_new: Optional[torch.Tensor], u_pos: torch.Tensor, u_cu: torch.Tensor, r_rank: torch.Tensor,
+                      r_cu_layer: torch.Tensor, max_ctx: Sequence[int], k_ctx_out: torch.Tensor,
+                      v_ctx_out: torch.Tensor, stream=None) -> None:
+    _check(lib().relaxkv_gather_kv(shape.ref(), int(mode), cache.ref(), _ptr(k_new), _ptr(v_new), _ptr(u_pos),
+                                   _ptr(u_cu), _ptr(r_rank), _ptr(r_cu_layer), _i32(max_ctx), _ptr(k_ctx_out),
+                                   _ptr(v_ctx_out), ctypes.c_int64(k_ctx_out.shape[0]), _stream(stream)),
+           "relaxkv_gather_kv")
+
+
+def relaxkv_read_device_status(stream=None):
+    """Synchronises the stream; returns (status, [kernel id, block, v0, v1]) and clears the word."""
+    st = ctypes.c_int32(0)
+    detail = (ctypes.c_int32 * 4)()
+    _check(lib().relaxkv_read_device_status(ctypes.byref(st), detail, _stream(stream)), "relaxkv_read_device_status")
+    return int(st.value), list(detail)

@@ -1,0 +1,73 @@
+// Host-side entry points that launch nothing heavy: status word, strings, anchor count, workspace size.
+#include <cfenv>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace relaxkv {
+
+__device__ DeviceStatus g_status_word;
+
+DeviceStatus* status_word() {
+  // One lookup per device; the address of a __device__ variable differs between devices.
+  static DeviceStatus* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<DeviceStatus*>(p);
+  }
+  return cached[dev];
+}
+
+}  // namespace relaxkv
+
+using namespace relaxkv;
+
+extern "C" const char* relaxkv_status_string(int32_t status) {
+  switch (status) {
+    case RELAXKV_OK: return "ok";
+    case RELAXKV_ERR_INVALID_ARG: return "invalid argument";
+    case RELAXKV_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case RELAXKV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case RELAXKV_ERR_CUDA: return "CUDA error";
+    case RELAXKV_ERR_BAD_INDEX: return "bad index seen on the device";
+    case RELAXKV_ERR_TIMEOUT: return "bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int32_t relaxkv_anchor_count(int32_t ctx_len, double ratio) {
+  if (ctx_len < 1) return 0;
+  const int old = std::fegetround();
+  std::fesetround(FE_TONEAREST);
+  double x = std::nearbyint(ratio * static_cast<double>(ctx_len));
+  std::fesetround(old);
+  long long k = static_cast<long long>(x);
+  if (k < 1) k = 1;
+  if (k > ctx_len) k = ctx_len;
+  return static_cast<int32_t>(k);
+}
+
+extern "C" size_t relaxkv_workspace_bytes(const relaxkv_shape* shape, int32_t n_layers, const int32_t* /*h_k*/) {
+  if (check_shape(shape) != RELAXKV_OK || n_layers < 1) return 0;
+  return ws_layout(shape, n_layers).total;
+}
+
+extern "C" relaxkv_status relaxkv_read_device_status(int32_t* h_status_out, int32_t* h_detail_out,
+                                                     relaxkv_stream stream) {
+  if (!h_status_out) return RELAXKV_ERR_INVALID_ARG;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  DeviceStatus h{};
+  if (cudaMemcpyAsync(&h, st, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return RELAXKV_ERR_CUDA;
+  if (cudaMemsetAsync(st, 0, sizeof(h), s) != cudaSuccess) return RELAXKV_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return RELAXKV_ERR_CUDA;
+  *h_status_out = h.status;
+  if (h_detail_out) {
+    h_detail_out[0] = h.kernel; h_detail_out[1] = h.block; h_detail_out[2] = h.v0; h_detail_out[3] = h.v1;
+  }
+  return RELAXKV_OK;
+}

@@ -1,0 +1,173 @@
+// Shared host/device helpers of the RelaxKV CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "relaxkv.h"
+
+namespace relaxkv {
+
+// ---- device status word -----------------------------------------------------------------
+// One int4 per device: {status, kernel id, block, value}.  Kernels record the first problem they
+// see with an atomic compare-and-swap and carry on without touching the offending data.
+struct DeviceStatus {
+  int status;
+  int kernel;
+  int block;
+  int v0;
+  int v1;
+};
+
+// Device address of the status word of the current device (defined in api.cu).
+DeviceStatus* status_word();
+
+enum KernelId : int {
+  KID_SETS = 1, KID_SELECT = 2, KID_SCORE = 3, KID_GATHER = 4, KID_SCATTER = 5,
+  KID_ATTN_SIMT = 6, KID_ATTN_SM100 = 7, KID_SCORE_SM100 = 8
+};
+
+__device__ __forceinline__ void report(DeviceStatus* st, int status, int kernel, int v0, int v1) {
+  if (atomicCAS(&st->status, 0, status) == 0) {
+    st->kernel = kernel;
+    st->block = (int)blockIdx.x;
+    st->v0 = v0;
+    st->v1 = v1;
+  }
+}
+
+// ---- host-side checks -------------------------------------------------------------------
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline relaxkv_status check_shape(const relaxkv_shape* s) {
+  if (!s || !s->h_ctx_len) return RELAXKV_ERR_INVALID_ARG;
+  if (s->n_req < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1) return RELAXKV_ERR_INVALID_ARG;
+  if (s->n_q_heads % s->n_kv_heads != 0) return RELAXKV_ERR_INVALID_ARG;
+  if (s->head_dim != 64 && s->head_dim != 128) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (s->n_q_heads / s->n_kv_heads > 16) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (s->n_req > 64) return RELAXKV_ERR_UNSUPPORTED_SHAPE;   // per-request scalars travel by value
+  for (int b = 0; b < s->n_req; ++b)
+    if (s->h_ctx_len[b] < 1) return RELAXKV_ERR_INVALID_ARG;
+  if (!(s->softmax_scale > 0.f)) return RELAXKV_ERR_INVALID_ARG;
+  return RELAXKV_OK;
+}
+
+inline relaxkv_status check_cache(const relaxkv_shape* s, const relaxkv_cache_view* c, bool need_v) {
+  if (!c || !c->k || (need_v && !c->v) || !c->h_req_token_offset) return RELAXKV_ERR_INVALID_ARG;
+  if (!aligned16(c->k) || (need_v && !aligned16(c->v))) return RELAXKV_ERR_INVALID_ARG;
+  if (c->token_stride < s->head_dim || c->head_stride < s->head_dim) return RELAXKV_ERR_INVALID_ARG;
+  if ((c->token_stride % 8) || (c->head_stride % 8)) return RELAXKV_ERR_INVALID_ARG;
+  for (int b = 0; b < s->n_req; ++b)
+    if (c->h_req_token_offset[b] < 0) return RELAXKV_ERR_INVALID_ARG;
+  return RELAXKV_OK;
+}
+
+inline relaxkv_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? RELAXKV_OK : RELAXKV_ERR_CUDA; }
+inline relaxkv_status launch_ok() { return cuda_ok(cudaGetLastError()); }
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Up to this many requests have their per-request scalars passed by value in kernel parameters.
+constexpr int kMaxReqInline = 64;
+
+// Per-request scalars a kernel needs, by value (small batches) - avoids any host->device copy.
+struct ReqTable {
+  int n_req;
+  int ctx_len[kMaxReqInline];
+  int q_len[kMaxReqInline];
+  int q_cu[kMaxReqInline + 1];      // prefix of q_len
+  long long ctx_cu[kMaxReqInline + 1];  // prefix of ctx_len
+  long long tok_off[kMaxReqInline];     // cache token offset
+  int k[kMaxReqInline];
+  int k_cu[kMaxReqInline + 1];
+  int bound_a[kMaxReqInline];       // call-specific host bound (e.g. max targets)
+  int bound_b[kMaxReqInline];       // call-specific host bound (e.g. max ctx)
+  int tile_cu[kMaxReqInline + 1];   // call-specific prefix (e.g. q tiles)
+};
+
+// Fills the shape-derived fields of a ReqTable (host).
+inline void fill_req_table(ReqTable& t, const relaxkv_shape* s, const relaxkv_cache_view* c, const int32_t* h_k) {
+  t.n_req = s->n_req;
+  t.q_cu[0] = 0; t.ctx_cu[0] = 0; t.k_cu[0] = 0; t.tile_cu[0] = 0;
+  for (int b = 0; b < s->n_req; ++b) {
+    t.ctx_len[b] = s->h_ctx_len[b];
+    t.q_len[b] = s->h_q_len ? s->h_q_len[b] : 0;
+    t.q_cu[b + 1] = t.q_cu[b] + t.q_len[b];
+    t.ctx_cu[b + 1] = t.ctx_cu[b] + t.ctx_len[b];
+    t.tok_off[b] = c ? c->h_req_token_offset[b] : 0;
+    t.k[b] = h_k ? h_k[b] : 0;
+    t.k_cu[b + 1] = t.k_cu[b] + t.k[b];
+    t.bound_a[b] = 0; t.bound_b[b] = 0; t.tile_cu[b + 1] = 0;
+  }
+}
+
+// ---- workspace layout -------------------------------------------------------------------
+// Calls are stream-ordered, so the regions of different calls overlap.
+constexpr int kScoreSplits = 16;      // key-range splits of the row-statistics pass
+constexpr int kCtxPadRows = 128;      // zero rows after the materialised context
+
+struct WsLayout {
+  // attention: materialised mixed context K~ / V~  [ctx_rows_cap, H_kv, D] bf16
+  size_t kctx, vctx; long long ctx_rows_cap;
+  // scoring: lse [H, sumQ] f32 | part [kScoreSplits, H, sumQ] float2 | colpart [H_kv, sumT] f32
+  size_t lse, part, colpart;
+  // sets: counts [B + L*B] i32
+  size_t counts;
+  size_t total;
+};
+
+inline WsLayout ws_layout(const relaxkv_shape* s, int n_layers) {
+  WsLayout w{};
+  long long sum_t = 0, sum_q = 0;
+  for (int b = 0; b < s->n_req; ++b) { sum_t += s->h_ctx_len[b]; sum_q += s->h_q_len ? s->h_q_len[b] : 0; }
+  const size_t row_bytes = (size_t)s->n_kv_heads * s->head_dim * 2;
+  w.ctx_rows_cap = sum_t + kCtxPadRows;
+  size_t a = 0;
+  w.kctx = a; a = align_up(a + (size_t)w.ctx_rows_cap * row_bytes, 1024);
+  w.vctx = a; a = align_up(a + (size_t)w.ctx_rows_cap * row_bytes, 1024);
+  size_t attn_total = a;
+  a = 0;
+  w.lse = a; a = align_up(a + (size_t)s->n_q_heads * sum_q * 4, 256);
+  w.part = a; a = align_up(a + (size_t)kScoreSplits * s->n_q_heads * sum_q * 8, 256);
+  w.colpart = a; a = align_up(a + (size_t)s->n_kv_heads * sum_t * 4, 256);
+  size_t score_total = a;
+  w.counts = 0;
+  size_t sets_total = align_up((size_t)(s->n_req + (size_t)n_layers * s->n_req + 2) * 4, 256);
+  w.total = attn_total > score_total ? attn_total : score_total;
+  if (sets_total > w.total) w.total = sets_total;
+  return w;
+}
+
+// ---- small device helpers -----------------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+
+__device__ __forceinline__ int warp_reduce_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_reduce_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_reduce_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_reduce_min(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Find the request that owns global tile/row index x given an inclusive-exclusive prefix array.
+__device__ __forceinline__ int find_segment(const int* cu, int n, int x) {
+  int b = 0;
+  while (b + 1 < n && x >= cu[b + 1]) ++b;
+  return b;
+}
+
+}  // namespace relaxkv

@@ -1,0 +1,332 @@
+"""GPU parity: every C-ABI call against the fp64 CPU oracle on the same seeded bits.
+
+Tolerances (bf16 inputs, fp32 accumulation, P rounded to bf16 before P*V):
+  attention outputs  max-abs <= 2e-2, mean-abs <= 2e-3
+  raw scores         |gpu - ref| <= 1e-3 * ref + 1e-6 / T_c ;  normalised scores abs <= 1e-3
+  anchors            bit-exact when scores are fed in exactly; otherwise exact outside a 1e-3
+                     relative band around the k-th score
+  sets, gather, scatter: bit-exact
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import relaxkv_oracle as orc
+from paper_2609_33503_b200 import inputs
+from tests.harness import Case, attention_errors, bf16_to_f64, check_anchor_band
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+def B():
+    from paper_2609_33503_b200 import binding
+    return binding
+
+
+def assert_status_ok():
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (B().status_string(st), detail)
+
+
+def small_llama(n_layers=2, ctx=(2048,), q=(48,)):
+    return inputs.scaled_down(inputs.llama8b_16k(), ctx, q, n_layers=n_layers, chunk=256)
+
+
+def small_qwen(n_layers=3, ctx=(1536,), q=(40,)):
+    return inputs.scaled_down(inputs.qwen14b_32k("calibrated"), ctx, q, n_layers=n_layers, chunk=128)
+
+
+def small_ragged():
+    return inputs.scaled_down(inputs.qwen14b_32k("calibrated"), (640, 1280, 2176), (17, 33, 64), n_layers=2, chunk=128)
+
+
+WORKLOADS = {
+    "tiny": inputs.tiny,
+    "llama_small": small_llama,
+    "qwen_small": small_qwen,
+    "ragged_small": small_ragged,
+}
+
+
+@pytest.fixture(scope="module", params=list(WORKLOADS))
+def case(request):
+    return Case(WORKLOADS[request.param]())
+
+
+# ------------------------------------------------------------------------- selection ----
+
+def test_scores_and_anchors(case):
+    w = case.w
+    s = case.make_session(want_norm=True)
+    s.score_select(case.q_layers, case.cache_views())
+    assert_status_ok()
+    raw = s.raw.cpu().numpy().astype(np.float64)
+    norm = s.norm.cpu().numpy().astype(np.float64)
+    anchors = s.anchors.cpu().numpy()
+    for l in range(w.n_layers):
+        for b in range(w.n_req):
+            T = w.ctx_lens[b]
+            ref = case.raw[(l, b)]
+            got = raw[l, case.ctx_cu[b]:case.ctx_cu[b + 1]]
+            assert np.all(np.abs(got - ref) <= 1e-3 * ref + 1e-6 / T), np.abs(got / ref - 1).max()
+            assert abs(got.sum() - 1.0) < 1e-3
+            np.testing.assert_allclose(norm[l, case.ctx_cu[b]:case.ctx_cu[b + 1]], orc.minmax(ref), atol=1e-3)
+            check_anchor_band(ref, case.k[b], anchors[l, case.k_cu[b]:case.k_cu[b + 1]])
+
+
+def test_scores_with_supplied_lse(case):
+    """Supplying the rows' log-normalisers skips the statistics pass and gives the same scores."""
+    w = case.w
+    s = case.make_session()
+    lses = []
+    for l in range(w.n_layers):
+        per_req = [orc.row_lse(case.req_q(l, b), case.req_k(l, b), case.scale) for b in range(w.n_req)]
+        lses.append(torch.from_numpy(np.concatenate(per_req, axis=1).astype(np.float32)).contiguous().to(case.device))
+    s.score_select(case.q_layers, case.cache_views(), row_lse_layers=lses)
+    assert_status_ok()
+    raw = s.raw.cpu().numpy().astype(np.float64)
+    for l in range(w.n_layers):
+        for b in range(w.n_req):
+            ref = case.raw[(l, b)]
+            got = raw[l, case.ctx_cu[b]:case.ctx_cu[b + 1]]
+            assert np.all(np.abs(got - ref) <= 1e-3 * ref + 1e-6 / w.ctx_lens[b])
+
+
+def test_select_exact_on_given_scores(case):
+    """Oracle scores rounded to fp32 go in; anchors must match the oracle's top-k of those very
+    values bit for bit (ties included: a block of equal scores is planted)."""
+    w = case.w
+    nb, L = w.n_req, w.n_layers
+    shape = case.make_session().shape
+    raw32 = np.zeros((L, int(case.ctx_cu[-1])), dtype=np.float32)
+    for l in range(L):
+        for b in range(nb):
+            r = case.raw[(l, b)].astype(np.float32)
+            kth = np.sort(r)[::-1][case.k[b] - 1]
+            idx = np.argsort(np.abs(r - kth))[:9]        # make 9 scores tie with the k-th one
+            r[idx] = kth
+            raw32[l, case.ctx_cu[b]:case.ctx_cu[b + 1]] = r
+    d_raw = torch.from_numpy(raw32).to(case.device)
+    d_anchor = torch.full((L, int(case.k_cu[-1])), -1, dtype=torch.int32, device=case.device)
+    d_norm = torch.empty_like(d_raw)
+    B().relaxkv_select_topk(shape, L, case.k, d_raw, d_anchor, norm_scores_out=d_norm)
+    assert_status_ok()
+    got = d_anchor.cpu().numpy()
+    for l in range(L):
+        for b in range(nb):
+            seg = raw32[l, case.ctx_cu[b]:case.ctx_cu[b + 1]].astype(np.float64)
+            np.testing.assert_array_equal(got[l, case.k_cu[b]:case.k_cu[b + 1]], orc.topk(seg, case.k[b]))
+            np.testing.assert_allclose(d_norm[l, case.ctx_cu[b]:case.ctx_cu[b + 1]].cpu().numpy(), orc.minmax(seg),
+                                       atol=2e-6)
+
+
+def test_active_sets_bitexact(case):
+    w = case.w
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    assert_status_ok()
+    n_u, n_r = s.counts()
+    u_cu = s.u_cu.cpu().numpy()
+    r_cu = s.r_cu.cpu().numpy()
+    u_pos, u_rank, h = s.u_pos.cpu().numpy(), s.u_rank.cpu().numpy(), s.highest_layer.cpu().numpy()
+    r_rank = s.r_rank.cpu().numpy()
+    for b in range(w.n_req):
+        ref = case.sets[b]
+        assert n_u[b] == len(ref.u_pos) == u_cu[b + 1] - u_cu[b]
+        np.testing.assert_array_equal(u_pos[u_cu[b]:u_cu[b + 1]], ref.u_pos)
+        np.testing.assert_array_equal(u_rank[case.ctx_cu[b]:case.ctx_cu[b + 1]], ref.u_rank)
+        np.testing.assert_array_equal(h[case.ctx_cu[b]:case.ctx_cu[b + 1]], ref.h)
+        prev = None
+        for l in range(w.n_layers):
+            i = l * w.n_req + b
+            got = r_rank[r_cu[i]:r_cu[i + 1]]
+            np.testing.assert_array_equal(got, ref.ranks(l))
+            assert n_r[l][b] == len(got)
+            if prev is not None:
+                assert set(got.tolist()) <= prev                     # monotone across layers
+            prev = set(got.tolist())
+
+
+# --------------------------------------------------------------------- gather / scatter ----
+
+@pytest.mark.parametrize("head_major", [False, True])
+def test_gather_and_scatter_bitexact(head_major):
+    case = Case(small_ragged(), head_major_cache=head_major)
+    w = case.w
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    nb = w.n_req
+    for l in range(w.n_layers):
+        f = case.fresh[l]
+        views = case.cache_views()
+        for mode in (B().CTX_UNION, B().CTX_FULL_PREFIX):
+            rows = (sum(case.max_ctx()) if mode == B().CTX_UNION else int(case.ctx_cu[-1])) + 64
+            kc = torch.full((rows, w.n_kv_heads, w.head_dim), 7.0, dtype=torch.bfloat16, device=case.device)
+            vc = torch.full_like(kc, 7.0)
+            s.gather(l, views[l], f.k_new, f.v_new, case.max_ctx(), kc, vc, mode=mode)
+            assert_status_ok()
+            kc_b, vc_b = inputs.bf16_bits(kc), inputs.bf16_bits(vc)
+            off = 0
+            for b in range(nb):
+                _, kn, vn = case.fresh_bits(l, b)
+                st = case.sets[b]
+                if mode == B().CTX_UNION:
+                    rk, rv = orc.mix_context(case.req_k(l, b), case.req_v(l, b), kn, vn, st.u_pos, st.ranks(l))
+                else:
+                    T = w.ctx_lens[b]
+                    rk, rv = orc.mix_context(case.req_k(l, b), case.req_v(l, b), kn, vn,
+                                             np.arange(T, dtype=np.int32), st.positions(l))
+                np.testing.assert_array_equal(kc_b[off:off + len(rk)], rk)
+                np.testing.assert_array_equal(vc_b[off:off + len(rv)], rv)
+                off += len(rk)
+            assert np.all(kc_b[off:off + 64] == 0) and np.all(vc_b[off:off + 64] == 0)     # zero pad rows
+        # scatter into a copy of the cache
+        k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+        if head_major:
+            k2 = case.k_cache[l].permute(1, 0, 2).contiguous().permute(1, 0, 2)
+            v2 = case.v_cache[l].permute(1, 0, 2).contiguous().permute(1, 0, 2)
+        view2 = B().CacheView(k2, v2, [int(x) for x in case.ctx_cu[:-1]])
+        for _ in range(2):                                            # idempotent
+            s.scatter(l, view2, f.k_new, f.v_new, case.max_targets(l))
+        assert_status_ok()
+        k2_b, v2_b = inputs.bf16_bits(k2), inputs.bf16_bits(v2)
+        for b in range(nb):
+            rk, rv = case.req_k(l, b).copy(), case.req_v(l, b).copy()
+            _, kn, vn = case.fresh_bits(l, b)
+            orc.scatter(rk, rv, kn, vn, case.sets[b].positions(l))
+            np.testing.assert_array_equal(k2_b[case.ctx_cu[b]:case.ctx_cu[b + 1]], rk)
+            np.testing.assert_array_equal(v2_b[case.ctx_cu[b]:case.ctx_cu[b + 1]], rv)
+
+
+# ---------------------------------------------------------------------------- attention ----
+
+def run_attention(case, s, l, mode, simt, use_fresh=True, views=None):
+    w = case.w
+    f = case.fresh[l]
+    out = torch.zeros_like(f.q_new)
+    lse = torch.zeros(w.n_q_heads, f.q_new.shape[0], dtype=torch.float32, device=case.device)
+    views = views or case.cache_views()
+    s.attention(l, views[l], f.q_new, f.k_new if use_fresh else None, f.v_new if use_fresh else None, out,
+                case.max_targets(l), case.max_ctx(), mode=mode, lse_out=lse, simt=simt)
+    assert_status_ok()
+    return out, lse
+
+
+def check_attention(case, l, out, lse, full_prefix, use_fresh=True):
+    f = case.fresh[l]
+    worst = (0.0, 0.0)
+    for b in range(case.w.n_req):
+        lo, hi = f.row_cu[b], f.row_cu[b + 1]
+        if hi == lo:
+            continue
+        ref, ref_lse = case.oracle_attention(l, b, full_prefix=full_prefix, use_fresh_kv=use_fresh)
+        mx, mean = attention_errors(out[lo:hi], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (l, b, mx, mean)
+        got_lse = lse[:, lo:hi].cpu().numpy().astype(np.float64).T
+        np.testing.assert_allclose(got_lse, ref_lse, atol=2e-3, rtol=1e-4)
+        worst = (max(worst[0], mx), max(worst[1], mean))
+    return worst
+
+
+@pytest.mark.parametrize("simt", [True, False], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("full_prefix", [False, True], ids=["union", "fullprefix"])
+def test_attention_matches_oracle(case, simt, full_prefix):
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    mode = B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION
+    for l in range(case.w.n_layers):
+        out, lse = run_attention(case, s, l, mode, simt)
+        check_attention(case, l, out, lse, full_prefix)
+
+
+def test_attention_orders_agree_and_is_deterministic(case):
+    """Update-then-attend from the cache equals mix-then-attend (Algorithm 1's order), bit for bit;
+    two runs give identical bits."""
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    l = case.w.n_layers - 1
+    f = case.fresh[l]
+    a, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
+    a2, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
+    assert torch.equal(a, a2)
+    k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+    view2 = B().CacheView(k2, v2, [int(x) for x in case.ctx_cu[:-1]])
+    s.scatter(l, view2, f.k_new, f.v_new, case.max_targets(l))
+    views = list(case.cache_views())
+    views[l] = view2
+    b_out, _ = run_attention(case, s, l, B().CTX_UNION, simt=False, use_fresh=False, views=views)
+    assert torch.equal(a, b_out)
+
+
+def test_full_ratio_is_dense_causal_attention():
+    """Anchor ratio 100 %: every position is an anchor at every layer, so the output must equal plain
+    causal attention over the fresh K/V (library SDPA in fp32 on the GPU, fp64 oracle on the CPU)."""
+    w = small_llama(n_layers=1, ctx=(700,), q=(8,)).replace(ratio=1.0)
+    case = Case(w)
+    assert case.k == [700]
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    out, lse = run_attention(case, s, 0, B().CTX_UNION, simt=False)
+    check_attention(case, 0, out, lse, False)
+    f = case.fresh[0]
+    G = w.group
+    q = f.q_new.float().permute(1, 0, 2).unsqueeze(0)
+    k = f.k_new.float().repeat_interleave(G, dim=1).permute(1, 0, 2).unsqueeze(0)
+    v = f.v_new.float().repeat_interleave(G, dim=1).permute(1, 0, 2).unsqueeze(0)
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, scale=case.scale)[0].permute(1, 0, 2)
+    d = (out.float() - ref).abs()
+    assert d.max().item() <= MAX_ABS and d.mean().item() <= MEAN_ABS
+
+
+@pytest.mark.parametrize("ctx,q,ratio", [((1,), (1,), 0.15), ((129,), (3,), 0.01), ((257,), (5,), 1.0), ((130, 1, 515), (2, 1, 7), 0.3)])
+def test_edge_sizes(ctx, q, ratio):
+    w = inputs.scaled_down(inputs.qwen14b_32k("literal"), ctx, q, n_layers=2, chunk=64).replace(ratio=ratio)
+    case = Case(w)
+    s = case.make_session(want_norm=True)
+    s.score_select(case.q_layers, case.cache_views())
+    assert_status_ok()
+    anchors = s.anchors.cpu().numpy()
+    for l in range(w.n_layers):
+        for b in range(w.n_req):
+            check_anchor_band(case.raw[(l, b)], case.k[b], anchors[l, case.k_cu[b]:case.k_cu[b + 1]])
+    s.build_active_sets(case.anchors_tensor())
+    for l in range(w.n_layers):
+        for full_prefix in (False, True):
+            out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
+            check_attention(case, l, out, lse, full_prefix)
+
+
+def test_loose_host_bounds_give_the_same_result(case):
+    """Host bounds may be loose (|R_l| <= |U| <= T_c): same bits as with exact bounds."""
+    w = case.w
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    l = 0
+    f = case.fresh[l]
+    exact, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
+    out = torch.zeros_like(f.q_new)
+    s.attention(l, case.cache_views()[l], f.q_new, f.k_new, f.v_new, out, list(w.ctx_lens), list(w.ctx_lens))
+    assert_status_ok()
+    assert torch.equal(out, exact)
+
+
+def test_bad_index_lists_are_reported_not_faulted():
+    """Out-of-range ranks are caught on the device: the status word says so, nothing faults."""
+    case = Case(small_llama(n_layers=1, ctx=(512,), q=(8,)))
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    torch.cuda.synchronize()
+    s.r_rank[:4] = torch.tensor([100000, -5, 100001, 100002], dtype=torch.int32, device=case.device)
+    f = case.fresh[0]
+    out = torch.zeros_like(f.q_new)
+    s.attention(0, case.cache_views()[0], f.q_new, f.k_new, f.v_new, out, case.max_targets(0), case.max_ctx())
+    st, detail = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX, (st, detail)
+    st, _ = B().relaxkv_read_device_status()
+    assert st == 0                                                  # reading clears the word
+    k2, v2 = case.k_cache[0].clone(), case.v_cache[0].clone()
+    s.scatter(0, B().CacheView(k2, v2, [0]), f.k_new, f.v_new, case.max_targets(0))
+    st, _ = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX
