@@ -161,6 +161,32 @@ relaxkv_status relaxkv_build_active_sets(
     void* workspace, size_t workspace_bytes, relaxkv_stream stream);
 
 /*
+ * relaxkv_build_active_sets for callers that have no scratch memory to give.  (The paper has no
+ * counterpart; this is a packaging variant of the call above and computes the same outputs.)
+ *
+ * Who needs it: code that runs inside a host which owns all device memory and lends an extension
+ * only its input and output tensors - an inference-server plug-in, an embedded runtime whose
+ * memory pool is sealed after start-up.  Such a caller can neither allocate a workspace nor ask
+ * its host for one.  Here the scratch (the B + n_layers*B set counts) lives in a fixed array inside
+ * the library image; the call allocates nothing and takes no workspace.  Inputs and outputs are
+ * still the caller's buffers, exactly as above.
+ *
+ * Limits and rules:
+ *  - B + n_layers*B must not exceed 8192 entries (32 KB, held by every GPU that loads the
+ *    library until the process exits); larger problems get RELAXKV_ERR_UNSUPPORTED_SHAPE.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing
+ *    in it needs to start at zero (each call overwrites every entry it later reads), but two calls
+ *    that overlap on the GPU - different streams, no ordering between them - race on it: order them.
+ *  - h_counts_pinned (optional) is filled from the array by a copy on `stream`, as above.
+ */
+relaxkv_status relaxkv_build_active_sets_static(
+    const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
+    int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
+    int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned, relaxkv_stream stream);
+
+/*
  * Sparse-context repair attention of one layer (Section 3.3, C_l(p); Section 3.4, mixed
  * fresh/cached K/V; Algorithm 1, steps 16-19; Appendix A.2).
  *

@@ -23,6 +23,7 @@ ENTRY_POINTS = (
     "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
+    "relaxkv_build_active_sets_static",
 )
 
 
@@ -178,6 +179,20 @@ def relaxkv_build_active_sets(shape: Shape, n_layers: int, k: Sequence[int], anc
                                            ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                            _stream(stream)),
            "relaxkv_build_active_sets")
+
+
+def relaxkv_build_active_sets_static(shape: Shape, n_layers: int, k: Sequence[int], anchors: torch.Tensor,
+                                     highest_layer_out: torch.Tensor, u_pos_out: torch.Tensor,
+                                     u_cu_out: torch.Tensor, u_rank_out: torch.Tensor, r_rank_out: torch.Tensor,
+                                     r_cu_out: torch.Tensor, counts_pinned: Optional[torch.Tensor] = None,
+                                     stream=None) -> None:
+    """Same outputs as relaxkv_build_active_sets, for callers that cannot supply a workspace: the
+    scratch is a fixed array inside the library (at most 8192 counts: n_req * (1 + n_layers))."""
+    _check(lib().relaxkv_build_active_sets_static(shape.ref(), int(n_layers), _i32(k), _ptr(anchors),
+                                                  _ptr(highest_layer_out), _ptr(u_pos_out), _ptr(u_cu_out),
+                                                  _ptr(u_rank_out), _ptr(r_rank_out), _ptr(r_cu_out),
+                                                  _ptr(counts_pinned), _stream(stream)),
+           "relaxkv_build_active_sets_static")
 
 
 def _attention(fn_name, shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, max_targets,
