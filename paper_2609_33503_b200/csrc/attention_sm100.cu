@@ -7,8 +7,10 @@
 //   softmax warps: tcgen05.ld S, position-based causal mask on the staircase edge, online max/sum with
 //                  lazy rescaling, P -> bf16 back into TMEM (over S)
 //   O += P V            (tcgen05.mma, A operand = P from TMEM, B = V tile MN-major from shared memory)
-// Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner.  Every wait is bounded; an expired wait raises the block's abort
+// A CTA runs TWO such query tiles (A, B) in ping-pong: while the softmax warps of one tile work, the
+// tensor pipe runs the other tile's MMAs; both tiles share every K/V tile staged in shared memory.
+// Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = query row = TMEM
+// lane), warp 8 TMA producer, warp 9 MMA issuer and TMEM owner.  Every wait is bounded; an expired wait raises the block's abort
 // flag, records RELAXKV_ERR_TIMEOUT in the device status word and the block tears down normally.
 #include "attention_common.cuh"
 #include "sm100_ptx.cuh"
@@ -24,21 +26,20 @@ constexpr float kRescaleThreshold = 8.0f;     // log2 units: rescale O only when
 constexpr int kBM = 128;                      // query rows per tile (TMEM lanes)
 constexpr int kBN = 128;                      // keys per context tile
 constexpr int kHalfBytes = 128 * 128;         // 128 rows x 64 bf16: one 128B-swizzled half tile
-constexpr int kStages = 2;
-constexpr int kAttnThreads = 192;
+constexpr int kRing = 5;                      // K/V tile buffers, used in the order K0 V0 K1 V1 ...
+constexpr int kAttnThreads = 384;             // 2 x 4 softmax warps + a control warpgroup (TMA warp, MMA warp, 2 idle)
 
 template <int D>
 struct AttnSmem {
   static constexpr int kHalves = D / 64;
   static constexpr int kTileBytes = kHalves * kHalfBytes;
-  static constexpr int kQ = 0;
-  static constexpr int kK = kQ + kTileBytes;
-  static constexpr int kV = kK + kStages * kTileBytes;
-  static constexpr int kBar = kV + kStages * kTileBytes;      // mbarriers (8 B each)
-  static constexpr int kNumBars = 4 + 3 * kStages;
-  static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem address, abort flag
+  static constexpr int kQ = 0;                                  // two query tiles
+  static constexpr int kKV = kQ + 2 * kTileBytes;               // ring of kRing K/V tiles
+  static constexpr int kBar = kKV + kRing * kTileBytes;         // mbarriers (8 B each)
+  static constexpr int kNumBars = 1 + 6 + 2 * kRing;
+  static constexpr int kMisc = kBar + 8 * kNumBars;             // tmem address, abort flag
   static constexpr int kTotal = kMisc + 16;
-  static constexpr int kDynamic = kTotal + 1024;              // slack to align the base to 1024 B
+  static constexpr int kDynamic = kTotal + 1024;                // slack to align the base to 1024 B
 };
 
 template <int D>
@@ -52,72 +53,85 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        DeviceStatus* st) {
   using L = AttnSmem<D>;
   constexpr int kHalves = L::kHalves;
-  constexpr uint32_t kTmemCols = (D == 128) ? 256u : 256u;   // S: 128 columns, O: D columns
-  constexpr uint32_t kColS = 0, kColO = 128;
+  constexpr uint32_t kTmemCols = 512;          // S_A | S_B | O_A | O_B, 128 columns each (O uses D of them)
 
-  // ---- which tile ------------------------------------------------------------------------------
+  // ---- which pair of query tiles ------------------------------------------------------------------
+  // rt.tile_cu counts tile PAIRS per request (from the host bounds); pairs are walked from the end of
+  // the target list (longest context first).  Tile A = the earlier targets, tile B = the later ones.
   const int B = rt.n_req;
   const int G = H / Hkv;
-  const int n_tiles_total = rt.tile_cu[B];
-  const int hd = blockIdx.x / n_tiles_total;                  // KV head (outermost: one head's K/V stays in L2)
-  const int tt = blockIdx.x - hd * n_tiles_total;
+  const int n_pairs_total = rt.tile_cu[B];
+  const int hd = blockIdx.x / n_pairs_total;                  // KV head outermost: its K/V stays in L2
+  const int tt = blockIdx.x - hd * n_pairs_total;
   const int b = find_segment(rt.tile_cu, B, tt);
-  const int t_rev = tt - rt.tile_cu[b];
+  const int p_rev = tt - rt.tile_cu[b];
   const int nr = r_cu[b + 1] - r_cu[b];
   const int nu = u_cu[b + 1] - u_cu[b];
-  const int n_tiles_true = (nr + tile_targets - 1) / tile_targets;
-  if (t_rev >= n_tiles_true) return;
+  const int pair_targets = 2 * tile_targets;
+  const int n_pairs_true = (nr + pair_targets - 1) / pair_targets;
+  if (p_rev >= n_pairs_true) return;
   if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b])) {
     if (threadIdx.x == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
     return;
   }
   if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;   // drain after a timeout
-  const int tile = n_tiles_true - 1 - t_rev;                  // longest tiles first
-  const int rho0 = tile * tile_targets;
-  const int n_valid = min(tile_targets, nr - rho0);
-  const long long q_row0 = (long long)(r_cu[b] - r_cu[0]) + rho0;
+  const int pair = n_pairs_true - 1 - p_rev;
+  const int rho0 = pair * pair_targets;                       // first target of tile A
   const int ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
   const long long ctx_base = (mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b];
-  // causal limit of the last target of the tile -> number of context tiles
-  int lim_last;
-  {
-    const int c = r_rank[r_cu[b] + rho0 + n_valid - 1];
-    const int cc = min(max(c, 0), max(nu - 1, 0));
-    lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[u_cu[b] + cc];
-    lim_last = min(max(lim_last, 0), ctx_len_b - 1);
+  const long long q_row_base = (long long)(r_cu[b] - r_cu[0]) + rho0;
+  // valid targets and context tiles of each query tile
+  int n_valid[2], n_kv[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    n_valid[x] = max(0, min(tile_targets, nr - rho0 - x * tile_targets));
+    n_kv[x] = 0;
+    if (n_valid[x] > 0) {
+      const int c = r_rank[r_cu[b] + rho0 + x * tile_targets + n_valid[x] - 1];
+      const int cc = min(max(c, 0), max(nu - 1, 0));
+      int lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[u_cu[b] + cc];
+      lim_last = min(max(lim_last, 0), ctx_len_b - 1);
+      n_kv[x] = lim_last / kBN + 1;
+    }
   }
-  const int n_kv = lim_last / kBN + 1;
+  const int n_kv_max = max(n_kv[0], n_kv[1]);
 
   // ---- shared memory -----------------------------------------------------------------------------
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base + L::kQ, k_smem = base + L::kK, v_smem = base + L::kV;
+  const uint32_t q_smem = base + L::kQ, kv_smem = base + L::kKV;
   const uint32_t bar0 = base + L::kBar;
-  const uint32_t bar_q = bar0, bar_sfull = bar0 + 8, bar_pfull = bar0 + 16, bar_odone = bar0 + 24;
-  const uint32_t bar_kfull = bar0 + 32, bar_vfull = bar_kfull + 8 * kStages, bar_empty = bar_vfull + 8 * kStages;
+  const uint32_t bar_q = bar0;
+  const uint32_t bar_sfull = bar0 + 8;          // [2]
+  const uint32_t bar_pfull = bar0 + 24;         // [2]
+  const uint32_t bar_ofinal = bar0 + 40;        // [2]
+  const uint32_t bar_full = bar0 + 56;          // [kRing]
+  const uint32_t bar_empty = bar_full + 8 * kRing;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_q, 1); mbar_init(bar_sfull, 1); mbar_init(bar_pfull, 128); mbar_init(bar_odone, 1);
-    for (int s = 0; s < kStages; ++s) { mbar_init(bar_kfull + 8 * s, 1); mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_q, 1);
+    for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
     tmem_relinquish();
   }
-  // rows of the Q tile that no (target, head) pair fills: zero them (they feed unused MMA rows)
+  // rows of the Q tiles that no (target, head) pair fills: zero them (they feed unused MMA rows)
   {
     const int used = tile_targets * G;
-    for (int i = threadIdx.x; i < (kBM - used) * 8 * kHalves; i += kAttnThreads) {
-      const int row = used + (i >> 3) % (kBM - used), piece = i & 7, half = (i >> 3) / (kBM - used);
-      *reinterpret_cast<uint4*>(base_ptr + L::kQ + half * kHalfBytes + row * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
+    const int n_pad = kBM - used;
+    for (int i = threadIdx.x; i < n_pad * 8 * kHalves * 2; i += kAttnThreads) {
+      const int piece = i & 7, r = (i >> 3) % n_pad, blk = (i >> 3) / n_pad;    // blk = tile * kHalves + half
+      *reinterpret_cast<uint4*>(base_ptr + L::kQ + blk * kHalfBytes + (used + r) * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
   }
@@ -126,64 +140,92 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 4) {
+  // Register budget: the control warpgroup gives registers to the two softmax warpgroups
+  // (12 warps x 168 at launch = 8 x 224 + 4 x 56).
+  if (warp >= 8) {
+  reg_dealloc<56>();
+  if (warp == 8) {
     // ================= TMA producer =================
     if (lane == 0) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      mbar_expect_tx(bar_q, (uint32_t)(kHalves * tile_targets * G * 128));
-      for (int hf = 0; hf < kHalves; ++hf)
-        tma_load_3d(q_smem + hf * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G, (int)q_row0);
-      for (int j = 0; j < n_kv; ++j) {
-        const int s = j % kStages;
-        if (j >= kStages && !mbar_wait(bar_empty + 8 * s, ((j / kStages) - 1) & 1, abort_flag)) break;
-        const int row = (int)(ctx_base + (long long)j * kBN);
-        mbar_expect_tx(bar_kfull + 8 * s, L::kTileBytes);
+      mbar_expect_tx(bar_q, (uint32_t)(2 * kHalves * tile_targets * G * 128));
+      for (int x = 0; x < 2; ++x)
         for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_3d(k_smem + s * L::kTileBytes + hf * kHalfBytes, &tm_k, bar_kfull + 8 * s, hf * 64, hd, row);
-        mbar_expect_tx(bar_vfull + 8 * s, L::kTileBytes);
+          tma_load_3d(q_smem + (x * kHalves + hf) * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G,
+                      (int)(q_row_base + x * tile_targets));
+      for (int u = 0; u < 2 * n_kv_max; ++u) {                // u = 2*j + (0: K, 1: V)
+        const int s = u % kRing;
+        if (u >= kRing && !mbar_wait(bar_empty + 8 * s, ((u / kRing) - 1) & 1, abort_flag)) break;
+        const int row = (int)(ctx_base + (long long)(u >> 1) * kBN);
+        const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
+        mbar_expect_tx(bar_full + 8 * s, L::kTileBytes);
         for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_3d(v_smem + s * L::kTileBytes + hf * kHalfBytes, &tm_v, bar_vfull + 8 * s, hf * 64, hd, row);
+          tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar_full + 8 * s, hf * 64, hd, row);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ================= MMA issuer =================
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kBM, kBN, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
-      const uint32_t t_s = tmem_base + kColS, t_o = tmem_base + kColO;
       bool ok = mbar_wait(bar_q, 0, abort_flag);
-      for (int j = 0; ok && j < n_kv; ++j) {
-        const int s = j % kStages;
-        const uint32_t ph = (j / kStages) & 1;
-        if (!(ok = mbar_wait(bar_kfull + 8 * s, ph, abort_flag))) break;
+      // S_x = Q_x K_j^T  -> bar_sfull[x]
+      auto issue_qk = [&](int x, int j) -> bool {
+        const int u = 2 * j, s = u % kRing;
+        if (!mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
         tc_fence_after();
+        const uint32_t qa = q_smem + x * L::kTileBytes, ka = kv_smem + s * L::kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          mma_ss(t_s, smem_desc_sw128(q_smem + off, 16, 1024),
-                 smem_desc_sw128(k_smem + s * L::kTileBytes + off, 16, 1024), idesc_qk, kk > 0);
+          mma_ss(tmem_base + x * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
+                 idesc_qk, kk > 0);
         }
-        mma_commit(bar_sfull);
-        if (!(ok = mbar_wait(bar_pfull, j & 1, abort_flag))) break;
-        if (!(ok = mbar_wait(bar_vfull + 8 * s, ph, abort_flag))) break;
+        mma_commit(bar_sfull + 8 * x);
+        return true;
+      };
+      // O_x += P_x V_j   (P_x read from TMEM where the softmax warps left it, over S_x)
+      auto issue_pv = [&](int x, int j) -> bool {
+        const int u = 2 * j + 1, s = u % kRing;
+        if (!mbar_wait(bar_pfull + 8 * x, j & 1, abort_flag)) return false;
+        if (!mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
         tc_fence_after();
+        const uint32_t va = kv_smem + s * L::kTileBytes;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {
-          mma_ts(t_o, t_s + kk * 8, smem_desc_sw128(v_smem + s * L::kTileBytes + kk * 2048, kHalfBytes, 1024),
-                 idesc_pv, (j > 0) || (kk > 0));
+        for (int kk = 0; kk < kBN / 16; ++kk)
+          mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + kk * 8,
+                 smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
+        if (j == n_kv[x] - 1) mma_commit(bar_ofinal + 8 * x);
+        return true;
+      };
+      if (ok && n_kv[0] > 0) ok = issue_qk(0, 0);
+      if (ok && n_kv[1] > 0) ok = issue_qk(1, 0);
+      if (ok) mma_commit(bar_empty + 8 * 0);                   // K_0's buffer: free once both S tiles are done
+      for (int j = 0; ok && j < n_kv_max; ++j) {
+        if (j < n_kv[0]) {
+          if (!(ok = issue_pv(0, j))) break;
+          if (j + 1 < n_kv[0] && !(ok = issue_qk(0, j + 1))) break;
         }
-        mma_commit(bar_empty + 8 * s);
-        mma_commit(bar_odone);
+        if (j < n_kv[1]) {
+          if (!(ok = issue_pv(1, j))) break;
+        }
+        mma_commit(bar_empty + 8 * ((2 * j + 1) % kRing));     // V_j
+        if (j + 1 < n_kv[1] && !(ok = issue_qk(1, j + 1))) break;
+        if (j + 1 < n_kv_max) mma_commit(bar_empty + 8 * ((2 * j + 2) % kRing));   // K_{j+1}
       }
     }
+  }
   } else {
+    reg_alloc<224>();
     // ================= softmax + epilogue: thread = query row = TMEM lane =================
-    const int row = threadIdx.x;                               // 0..127
+    const int x = warp >> 2;                                    // 0: tile A, 1: tile B
+    const int row = threadIdx.x & 127;
     const int t_local = row / G, j_head = row - t_local * G;
-    const bool row_valid = (row < tile_targets * G) && (t_local < n_valid);
+    const bool row_valid = (row < tile_targets * G) && (t_local < n_valid[x]);
+    const int rho_t = rho0 + x * tile_targets + t_local;
     int limit = 0;
     if (row_valid) {
-      const int c = r_rank[r_cu[b] + rho0 + t_local];
+      const int c = r_rank[r_cu[b] + rho_t];
       if (c < 0 || c >= nu) {
         report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
       } else {
@@ -191,12 +233,14 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (limit < 0 || limit >= ctx_len_b) { report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, limit, ctx_len_b); limit = 0; }
       }
     }
-    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-    const uint32_t t_s = lane_base + kColS, t_o = lane_base + kColO;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_s = lane_base + x * 128, t_o = lane_base + 256 + x * 128;
+    const uint32_t my_sfull = bar_sfull + 8 * x, my_pfull = bar_pfull + 8 * x;
+    const int my_n = n_kv[x];
     float m = -INFINITY, z = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      ok = mbar_wait(bar_sfull, j & 1, abort_flag);
+    for (int j = 0; j < my_n; ++j) {
+      ok = mbar_wait(my_sfull, j & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -217,12 +261,9 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (j == 0) {
         m = m_new;
       } else {
+        // S_x(j) is complete, hence so is O_x += P_x V_{j-1}: O_x may be rescaled here
         const bool need = m_new > m + kRescaleThreshold;
         if (__any_sync(0xffffffffu, need)) {
-          ok = mbar_wait(bar_odone, (j - 1) & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
           float alpha = 1.f;
           if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
 #pragma unroll
@@ -237,31 +278,33 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tmem_wait_st();
         }
       }
-      uint32_t pk[kBN / 2];
       float zs = 0.f;
 #pragma unroll
-      for (int i = 0; i < kBN; i += 2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(s[i]), scale_log2, -m));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(s[i + 1]), scale_log2, -m));
-        zs += p0 + p1;
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-        pk[i >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+      for (int c = 0; c < kBN / 32; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i]), scale_log2, -m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2, -m));
+          zs += p0 + p1;
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+          pk[i >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        tmem_st16(t_s + c * 16, pk);
       }
       z += zs;
-      tmem_st32(t_s, &pk[0]);
-      tmem_st32(t_s + 32, &pk[32]);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_pfull);
+      mbar_arrive(my_pfull);
     }
-    if (ok) {
-      ok = mbar_wait(bar_odone, (n_kv - 1) & 1, abort_flag);
+    if (ok && my_n > 0) {
+      ok = mbar_wait(bar_ofinal + 8 * x, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
     }
-    if (ok) {
+    if (ok && my_n > 0) {
       tc_fence_after();
       const float inv = 1.f / z;
-      const long long orow = q_row0 + t_local;
+      const long long orow = q_row_base + x * tile_targets + t_local;
       uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -290,13 +333,13 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, tile, hd);
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, pair, hd);
     // give copies and MMAs still in flight time to land before shared memory and TMEM are released
     const uint64_t t0 = global_timer_ns();
     while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
@@ -341,8 +384,8 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   const int H = shape->n_q_heads, Hkv = shape->n_kv_heads, G = H / Hkv;
   const int tile_targets = kBM / G;
   const int B = shape->n_req;
-  for (int b = 0; b < B; ++b)
-    plan.rt.tile_cu[b + 1] = plan.rt.tile_cu[b] + (plan.rt.bound_a[b] + tile_targets - 1) / tile_targets;
+  for (int b = 0; b < B; ++b)     // tile_cu counts PAIRS of query tiles
+    plan.rt.tile_cu[b + 1] = plan.rt.tile_cu[b] + (plan.rt.bound_a[b] + 2 * tile_targets - 1) / (2 * tile_targets);
   const long long grid = (long long)plan.rt.tile_cu[B] * Hkv;
   if (grid == 0) return RELAXKV_OK;
   if (grid > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
