@@ -104,13 +104,21 @@ inline void fill_req_table(ReqTable& t, const relaxkv_shape* s, const relaxkv_ca
 
 // ---- workspace layout -------------------------------------------------------------------
 // Calls are stream-ordered, so the regions of different calls overlap.
-constexpr int kScoreSplits = 16;      // key-range splits of the row-statistics pass
+constexpr int kScoreSplitsMax = 64;   // key-range splits of the scoring passes (grid.z), at most
+constexpr int kScoreMaxRows = 640;    // query rows (token x head-in-group) resident per scoring CTA
+constexpr int kScoreTokBox = 8;       // query tokens per TMA box of the scoring kernel
 constexpr int kCtxPadRows = 128;      // zero rows after the materialised context
+
+// Query-row blocks a request needs so that each block's rows fit resident (scoring kernel).
+inline int score_blocks(int q_len, int group) {
+  const int max_tok = kScoreMaxRows / group / kScoreTokBox * kScoreTokBox;
+  return q_len > 0 ? (q_len + max_tok - 1) / max_tok : 0;
+}
 
 struct WsLayout {
   // attention: materialised mixed context K~ / V~  [ctx_rows_cap, H_kv, D] bf16
   size_t kctx, vctx; long long ctx_rows_cap;
-  // scoring: lse [H, sumQ] f32 | part [kScoreSplits, H, sumQ] float2 | colpart [H_kv, sumT] f32
+  // scoring: lse [H, sumQ] f32 | part [2*kScoreSplitsMax, H, sumQ] float2 | colpart [2*H_kv*max_blocks, sumT] f32
   size_t lse, part, colpart;
   // sets: counts [B + L*B] i32
   size_t counts;
@@ -129,8 +137,13 @@ inline WsLayout ws_layout(const relaxkv_shape* s, int n_layers) {
   size_t attn_total = a;
   a = 0;
   w.lse = a; a = align_up(a + (size_t)s->n_q_heads * sum_q * 4, 256);
-  w.part = a; a = align_up(a + (size_t)kScoreSplits * s->n_q_heads * sum_q * 8, 256);
-  w.colpart = a; a = align_up(a + (size_t)s->n_kv_heads * sum_t * 4, 256);
+  int max_blocks = 1;
+  for (int b = 0; b < s->n_req; ++b) {
+    const int nb = score_blocks(s->h_q_len ? s->h_q_len[b] : 0, s->n_q_heads / s->n_kv_heads);
+    if (nb > max_blocks) max_blocks = nb;
+  }
+  w.part = a; a = align_up(a + (size_t)2 * kScoreSplitsMax * s->n_q_heads * sum_q * 8, 256);
+  w.colpart = a; a = align_up(a + (size_t)2 * s->n_kv_heads * max_blocks * sum_t * 4, 256);
   size_t score_total = a;
   w.counts = 0;
   size_t sets_total = align_up((size_t)(s->n_req + (size_t)n_layers * s->n_req + 2) * 4, 256);

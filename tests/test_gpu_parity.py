@@ -280,7 +280,8 @@ def test_full_ratio_is_dense_causal_attention():
     assert d.max().item() <= MAX_ABS and d.mean().item() <= MEAN_ABS
 
 
-@pytest.mark.parametrize("ctx,q,ratio", [((1,), (1,), 0.15), ((129,), (3,), 0.01), ((257,), (5,), 1.0), ((130, 1, 515), (2, 1, 7), 0.3)])
+@pytest.mark.parametrize("ctx,q,ratio", [((1,), (1,), 0.15), ((129,), (3,), 0.01), ((257,), (5,), 1.0), ((130, 1, 515), (2, 1, 7), 0.3),
+                                         ((1000, 300), (200, 131), 0.15)])
 def test_edge_sizes(ctx, q, ratio):
     w = inputs.scaled_down(inputs.qwen14b_32k("literal"), ctx, q, n_layers=2, chunk=64).replace(ratio=ratio)
     case = Case(w)
