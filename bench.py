@@ -54,6 +54,21 @@ def make_workload(args) -> inputs.Workload:
     raise SystemExit(f"unknown workload {args.workload}")
 
 
+def max_over_ranks(ms: float, device, world: int) -> float:
+    """Elapsed time of the slowest rank (the job's time); identity on one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Aggregate TFLOP/s over all ranks (each rank runs one replica of the workload)."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -168,6 +183,28 @@ class GpuJob:
         # kernels per step: per layer 4 scoring + gather + attention + scatter; 1 select; 5 for the sets
         self.launches_per_step = L * 7 + 1 + 5
 
+    def time_gather(self, mode):
+        """One pass over the layers of relaxkv_gather_kv alone (same kernel and arguments as inside the
+        attention call), CUDA events around each call; other layers' traffic keeps L2 cold."""
+        w, s = self.w, self.s
+        n_u, n_r = s.counts()
+        rows = (sum(n_u) if mode == self.B.CTX_UNION else int(self.ctx_cu[-1])) + 128
+        kc = torch.empty(rows, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device=self.device)
+        vc = torch.empty_like(kc)
+        total = 0.0
+        for rep in range(2):
+            evs = []
+            for l in range(w.n_layers):
+                f = self.fresh[l]
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                s.gather(l, self.views[l], f[1], f[2], n_u, kc, vc, mode=mode)
+                b_.record()
+                evs.append((a, b_))
+            torch.cuda.synchronize()
+            total = sum(a.elapsed_time(b_) for a, b_ in evs)
+        return total
+
     def flops(self, full_prefix=False):
         w = self.w
         e = sum(self.edges_full if full_prefix else self.edges)
@@ -216,11 +253,7 @@ def run_gpu(args):
     barrier()
     elapsed_ms = t0.elapsed_time(t1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([elapsed_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, device, world)
     st, detail = B.relaxkv_read_device_status()
     if st != 0:
         raise SystemExit(f"device status {B.status_string(st)} {detail}")
@@ -231,7 +264,10 @@ def run_gpu(args):
     phase_ms = {k: v / args.steps for k, v in phase_ms.items()}
     ms_per_step = elapsed_ms / args.steps
     flops = job.flops(args.full_prefix)
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(flops, world, ms_per_step)
+
+    # ---- the gather step on its own (it runs inside every attention call) -------------------------------
+    gather_ms = job.time_gather(mode)
 
     # ---- end-to-end arm: host buffers, copies inside the timed region --------------------------------
     e2e = None
@@ -245,6 +281,9 @@ def run_gpu(args):
     kv_row = w.n_kv_heads * w.head_dim * 2
     scatter_bytes = sum(2 * 2 * sum(nr) * kv_row for nr in job.n_r)          # K and V, read + write
     sum_t = int(job.ctx_cu[-1])
+    ctx_rows = sum(job.n_u) if not args.full_prefix else sum_t
+    gather_bytes = L * 2 * 2 * ctx_rows * kv_row                               # K and V, read + write
+    attn_kernel_ms = max(1e-9, phase_ms["attention"] - gather_ms)
     select_bytes = L * sum_t * w.n_kv_heads * w.head_dim * 2                  # each layer's K read once
     out = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -263,11 +302,15 @@ def run_gpu(args):
         "scatter_gbs": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9, 1),
         "scatter_frac_hbm": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
         "select_gbs": round(select_bytes / (phase_ms["score_select"] * 1e-3) / 1e9, 1),
+        "gather_us": round(gather_ms * 1e3, 1),
+        "gather_gbs": round(gather_bytes / (gather_ms * 1e-3) / 1e9, 1),
+        "gather_frac_hbm": round(gather_bytes / (gather_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
         "roofline": {"bound": "tensor", "achieved": round(attn_tflops, 2), "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": round(attn_tflops / peaks["bf16_tflops_sustained"], 4),
                      "frac_of_burst_peak": round(attn_tflops / peaks["bf16_tflops"], 4),
                      "traffic": None, "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
-                     "kernel": "attention_sm100_kernel (call time includes its gather launch)"},
+                     "kernel": "attention_sm100_kernel (timed per call, which includes its gather launch)",
+                     "achieved_without_gather": round(flops / (attn_kernel_ms * 1e-3) / 1e12, 2)},
         "clocks": clocks, "gpu_launches": job.launches_per_step * args.steps, "e2e": e2e,
     }
     if not args.no_cpu and world == 1:
@@ -306,12 +349,8 @@ def run_e2e(job, args, mode, world):
     t1.record()
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1) / n
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device=job.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return {"value": round(world * job.flops(args.full_prefix) / (ms * 1e-3) / 1e12, 3), "unit": UNIT,
+    ms = max_over_ranks(ms, job.device, world)
+    return {"value": round(whole_job_value(job.flops(args.full_prefix), world, ms), 3), "unit": UNIT,
             "ms_per_step": round(ms, 3), "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n}
 
 

@@ -254,9 +254,17 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int i = 0; i < kBN; ++i)
           if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
       }
-      float mx = -INFINITY;
+      // row maximum: eight independent chains instead of one 128-deep dependency chain
+      float mx8[8];
 #pragma unroll
-      for (int i = 0; i < kBN; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+      for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
+#pragma unroll
+      for (int i = 8; i < kBN; i += 8) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[i + e]));
+      }
+      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
       const float m_new = mx * scale_log2;
       if (j == 0) {
         m = m_new;
@@ -278,21 +286,24 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tmem_wait_st();
         }
       }
-      float zs = 0.f;
+      float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
 #pragma unroll
       for (int c = 0; c < kBN / 32; ++c) {
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
+        for (int i = 0; i < 32; i += 4) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i]), scale_log2, -m));
           const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2, -m));
-          zs += p0 + p1;
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-          pk[i >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+          const float p2 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2, -m));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2, -m));
+          zs0 += p0; zs1 += p1; zs2 += p2; zs3 += p3;
+          __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
+          pk[i >> 1] = *reinterpret_cast<uint32_t*>(&h01);
+          pk[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h23);
         }
         tmem_st16(t_s + c * 16, pk);
       }
-      z += zs;
+      z += (zs0 + zs1) + (zs2 + zs3);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(my_pfull);
