@@ -5,17 +5,27 @@
 
 namespace relaxkv {
 
-__device__ __forceinline__ int lower_bound_i32(const int* a, int n, int key) {
-  int lo = 0, hi = n;
-  while (lo < hi) {
-    int mid = (lo + hi) >> 1;
-    if (a[mid] < key) lo = mid + 1; else hi = mid;
+constexpr int kGatherRows = 8;            // one warp resolves the source of one context row
+constexpr int kGatherThreads = 256;
+
+// Warp-cooperative lower bound on an ascending list: 32 pivots per round instead of one.
+// Returns the first index with a[idx] >= key (n if none).  All lanes get the result.
+__device__ __forceinline__ int warp_lower_bound(const int* __restrict__ a, int n, int key, int lane) {
+  int lo = 0, hi = n;                     // the answer lies in [lo, hi]
+  while (hi > lo) {
+    const int step = (hi - lo + 31) / 32;
+    const int idx = lo + lane * step;
+    const bool lt = (idx < hi) && (__ldg(a + idx) < key);
+    const int n_lt = __popc(__ballot_sync(0xffffffffu, lt));   // pivots below the key: a prefix of the lanes
+    if (n_lt == 0) {
+      hi = lo;
+    } else {
+      hi = min(hi, lo + n_lt * step);
+      lo = lo + (n_lt - 1) * step + 1;
+    }
   }
   return lo;
 }
-
-constexpr int kGatherRows = 4;
-constexpr int kGatherThreads = 256;
 
 // One block moves kGatherRows context rows (all KV heads, K and V).
 // Context row x of request b is the fresh state of target rho if its context entry is an active
@@ -33,71 +43,85 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
   __shared__ int src_kind[kGatherRows];        // 0 = cache, 1 = fresh, 2 = zero fill, 3 = skip
   const long long row0 = (long long)blockIdx.x * kGatherRows;
   const int B = rt.n_req;
-  if (threadIdx.x < kGatherRows) {
-    const long long x = row0 + threadIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  {
+    const long long x = row0 + warp;
     int kind = 3;
     long long off = 0;
-    const long long total = (mode == RELAXKV_CTX_UNION) ? (long long)u_cu[B] : rt.ctx_cu[B];
+    const long long total = (mode == RELAXKV_CTX_UNION) ? (long long)__ldg(u_cu + B) : rt.ctx_cu[B];
     if (x < ctx_rows) {
       if (x >= total) {
         kind = (x < total + kCtxPadRows) ? 2 : 3;
       } else {
         int b = 0, c = -1, p;
         if (mode == RELAXKV_CTX_UNION) {
-          while (b + 1 < B && x >= u_cu[b + 1]) ++b;
-          c = (int)(x - u_cu[b]);
-          p = u_pos[x];
+          while (b + 1 < B && x >= __ldg(u_cu + b + 1)) ++b;
+          c = (int)(x - __ldg(u_cu + b));
+          p = __ldg(u_pos + x);
         } else {
           while (b + 1 < B && x >= rt.ctx_cu[b + 1]) ++b;
           p = (int)(x - rt.ctx_cu[b]);
-          const int nu = u_cu[b + 1] - u_cu[b];
-          const int lb = lower_bound_i32(u_pos + u_cu[b], nu, p);
-          if (lb < nu && u_pos[u_cu[b] + lb] == p) c = lb;
+          const int ub = __ldg(u_cu + b), nu = __ldg(u_cu + b + 1) - ub;
+          const int lb = warp_lower_bound(u_pos + ub, nu, p, lane);
+          if (lb < nu && __ldg(u_pos + ub + lb) == p) c = lb;
         }
         if (p < 0 || p >= rt.ctx_len[b]) {
-          report(st, RELAXKV_ERR_BAD_INDEX, KID_GATHER, (int)x, p);
+          if (lane == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_GATHER, (int)x, p);
           kind = 2;
         } else {
           kind = 0;
           off = (rt.tok_off[b] + p) * tok_stride;
           if (k_new != nullptr && c >= 0) {
-            const int nr = r_cu[b + 1] - r_cu[b];
-            const int rho = lower_bound_i32(r_rank + r_cu[b], nr, c);
-            if (rho < nr && r_rank[r_cu[b] + rho] == c) {
+            const int rb = __ldg(r_cu + b), nr = __ldg(r_cu + b + 1) - rb;
+            const int rho = warp_lower_bound(r_rank + rb, nr, c, lane);
+            if (rho < nr && __ldg(r_rank + rb + rho) == c) {
               kind = 1;
-              off = (long long)(r_cu[b] - r_cu[0] + rho) * n_kv_heads * head_dim;
+              off = (long long)(rb - __ldg(r_cu) + rho) * n_kv_heads * head_dim;
             }
           }
         }
       }
     }
-    src_kind[threadIdx.x] = kind;
-    src_off[threadIdx.x] = off;
+    if (lane == 0) { src_kind[warp] = kind; src_off[warp] = off; }
   }
   __syncthreads();
   const int pieces_per_head = head_dim / 8;                 // 16-byte pieces
   const int pieces_per_row = n_kv_heads * pieces_per_head;
   const int total_pieces = kGatherRows * pieces_per_row;
-  for (int i = threadIdx.x; i < total_pieces; i += kGatherThreads) {
-    const int r = i / pieces_per_row;
-    const int kind = src_kind[r];
-    if (kind == 3) continue;
-    const int pr = i - r * pieces_per_row;
-    const int g = pr / pieces_per_head;
-    const int part = pr - g * pieces_per_head;
-    const long long dst = ((row0 + r) * n_kv_heads + g) * head_dim + part * 8;
-    uint4 kk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-    if (kind == 0) {
-      const long long s = src_off[r] + g * head_stride + part * 8;
-      kk = __ldg(reinterpret_cast<const uint4*>(cache_k + s));
-      vv = __ldg(reinterpret_cast<const uint4*>(cache_v + s));
-    } else if (kind == 1) {
-      const long long s = src_off[r] + (long long)g * head_dim + part * 8;
-      kk = __ldg(reinterpret_cast<const uint4*>(k_new + s));
-      vv = __ldg(reinterpret_cast<const uint4*>(v_new + s));
+  for (int i0 = threadIdx.x; i0 < total_pieces; i0 += 4 * kGatherThreads) {
+    uint4 kk[4], vv[4];
+    long long dst[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {                            // issue every load before the first store
+      const int i = i0 + u * kGatherThreads;
+      kk[u] = make_uint4(0, 0, 0, 0); vv[u] = make_uint4(0, 0, 0, 0); dst[u] = -1;
+      if (i < total_pieces) {
+        const int r = i / pieces_per_row;
+        const int kind = src_kind[r];
+        if (kind != 3) {
+          const int pr = i - r * pieces_per_row;
+          const int g = pr / pieces_per_head;
+          const int part = pr - g * pieces_per_head;
+          dst[u] = ((row0 + r) * n_kv_heads + g) * head_dim + part * 8;
+          if (kind == 0) {
+            const long long so = src_off[r] + g * head_stride + part * 8;
+            kk[u] = __ldg(reinterpret_cast<const uint4*>(cache_k + so));
+            vv[u] = __ldg(reinterpret_cast<const uint4*>(cache_v + so));
+          } else if (kind == 1) {
+            const long long so = src_off[r] + (long long)g * head_dim + part * 8;
+            kk[u] = __ldg(reinterpret_cast<const uint4*>(k_new + so));
+            vv[u] = __ldg(reinterpret_cast<const uint4*>(v_new + so));
+          }
+        }
+      }
     }
-    *reinterpret_cast<uint4*>(k_out + dst) = kk;
-    *reinterpret_cast<uint4*>(v_out + dst) = vv;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (dst[u] >= 0) {
+        *reinterpret_cast<uint4*>(k_out + dst[u]) = kk[u];
+        *reinterpret_cast<uint4*>(v_out + dst[u]) = vv[u];
+      }
+    }
   }
 }
 
