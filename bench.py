@@ -29,6 +29,11 @@ import torch
 
 from paper_2609_33503_b200 import inputs
 
+# DRAM bytes per target row of the attention kernel, from the ncu capture summarised in
+# profiles/attention_sm100_qwen14b_32k_layer.md (dram read + write of one launch / its target rows);
+# traffic grows with the rows (Q in, O out), so a launch's traffic is this figure x its rows.
+ATTN_DRAM_BYTES_PER_TARGET_ROW_D128_H40 = 20200.0
+
 METRIC = "repair_attention_tflops"
 UNIT = "TFLOP/s"
 
@@ -284,6 +289,12 @@ def run_gpu(args):
     ctx_rows = sum(job.n_u) if not args.full_prefix else sum_t
     gather_bytes = L * 2 * 2 * ctx_rows * kv_row                               # K and V, read + write
     attn_kernel_ms = max(1e-9, phase_ms["attention"] - gather_ms)
+    traffic = None
+    if w.head_dim == 128 and w.n_q_heads == 40:      # the shape the capture was taken on
+        traffic = {"bytes_per_launch": round(ATTN_DRAM_BYTES_PER_TARGET_ROW_D128_H40 * sum(sum(x) for x in job.n_r) / L),
+                   "algorithmic_bytes_per_launch": round((2 * sum(sum(x) for x in job.n_r) * w.n_q_heads * w.head_dim * 2
+                                                          + 2 * ctx_rows * kv_row) / L),
+                   "how": "ncu dram read+write of one launch on a smaller capture, scaled by target rows"}
     select_bytes = L * sum_t * w.n_kv_heads * w.head_dim * 2                  # each layer's K read once
     out = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -308,7 +319,7 @@ def run_gpu(args):
         "roofline": {"bound": "tensor", "achieved": round(attn_tflops, 2), "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": round(attn_tflops / peaks["bf16_tflops_sustained"], 4),
                      "frac_of_burst_peak": round(attn_tflops / peaks["bf16_tflops"], 4),
-                     "traffic": None, "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
+                     "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
                      "kernel": "attention_sm100_kernel (timed per call, which includes its gather launch)",
                      "achieved_without_gather": round(flops / (attn_kernel_ms * 1e-3) / 1e12, 2)},
         "clocks": clocks, "gpu_launches": job.launches_per_step * args.steps, "e2e": e2e,
