@@ -36,7 +36,7 @@ struct AttnSmem {
   static constexpr int kQ = 0;                                  // two query tiles
   static constexpr int kKV = kQ + 2 * kTileBytes;               // ring of kRing K/V tiles
   static constexpr int kBar = kKV + kRing * kTileBytes;         // mbarriers (8 B each)
-  static constexpr int kNumBars = 1 + 6 + 2 * kRing;
+  static constexpr int kNumBars = 1 + 8 + 2 * kRing;
   static constexpr int kMisc = kBar + 8 * kNumBars;             // tmem address, abort flag
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                // slack to align the base to 1024 B
@@ -104,9 +104,10 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar0 = base + L::kBar;
   const uint32_t bar_q = bar0;
   const uint32_t bar_sfull = bar0 + 8;          // [2]
-  const uint32_t bar_pfull = bar0 + 24;         // [2]
-  const uint32_t bar_ofinal = bar0 + 40;        // [2]
-  const uint32_t bar_full = bar0 + 56;          // [kRing]
+  const uint32_t bar_pfull = bar0 + 24;         // [2] first 64 keys of P ready
+  const uint32_t bar_pfull_hi = bar0 + 40;      // [2] last 64 keys of P ready
+  const uint32_t bar_ofinal = bar0 + 56;        // [2]
+  const uint32_t bar_full = bar0 + 72;          // [kRing]
   const uint32_t bar_empty = bar_full + 8 * kRing;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
@@ -115,7 +116,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
+    for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_pfull_hi + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
     for (int s = 0; s < kRing; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     *abort_flag = 0;
     fence_barrier_init();
@@ -192,9 +193,16 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_after();
         const uint32_t va = kv_smem + s * L::kTileBytes;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)
+        for (int kk = 0; kk < kBN / 32; ++kk)
           mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + kk * 8,
                  smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
+        // the second half of P arrives while the first half is being multiplied
+        if (!mbar_wait(bar_pfull_hi + 8 * x, j & 1, abort_flag)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = kBN / 32; kk < kBN / 16; ++kk)
+          mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + kk * 8,
+                 smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_pv, 1u);
         if (j == n_kv[x] - 1) mma_commit(bar_ofinal + 8 * x);
         return true;
       };
@@ -302,11 +310,16 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           pk[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h23);
         }
         tmem_st16(t_s + c * 16, pk);
+        if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(my_pfull);
+        }
       }
       z += (zs0 + zs1) + (zs2 + zs3);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(my_pfull);
+      mbar_arrive(bar_pfull_hi + 8 * x);
     }
     if (ok && my_n > 0) {
       ok = mbar_wait(bar_ofinal + 8 * x, 0, abort_flag);
