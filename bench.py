@@ -292,8 +292,8 @@ def run_gpu(args):
     traffic = None
     if w.head_dim == 128 and w.n_q_heads == 40:      # the shape the capture was taken on
         traffic = {"bytes_per_launch": round(ATTN_DRAM_BYTES_PER_TARGET_ROW_D128_H40 * sum(sum(x) for x in job.n_r) / L),
-                   "algorithmic_bytes_per_launch": round((2 * sum(sum(x) for x in job.n_r) * w.n_q_heads * w.head_dim * 2
-                                                          + 2 * ctx_rows * kv_row) / L),
+                   "algorithmic_bytes_per_launch": round(2 * sum(sum(x) for x in job.n_r) / L * w.n_q_heads * w.head_dim * 2
+                                                         + 2 * ctx_rows * kv_row),
                    "how": "ncu dram read+write of one launch on a smaller capture, scaled by target rows"}
     select_bytes = L * sum_t * w.n_kv_heads * w.head_dim * 2                  # each layer's K read once
     out = {
