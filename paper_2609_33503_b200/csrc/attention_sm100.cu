@@ -171,54 +171,46 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       // S_x = Q_x K_j^T  -> bar_sfull[x]
-      auto issue_qk = [&](int x, int j) -> bool {
+      // (a successful mbarrier wait costs the issuing thread ~150 cycles, so a tile that is known to be
+      //  in shared memory - the other query tile already waited for it - is not waited for again)
+      auto issue_qk = [&](int x, int j, bool wait_tile) -> bool {
         const int u = 2 * j, s = u % kRing;
-        if (!mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
+        if (wait_tile && !mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t qa = q_smem + x * L::kTileBytes, ka = kv_smem + s * L::kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          mma_ss(tmem_base + x * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
-                 idesc_qk, kk > 0);
-        }
+        mma_ss_kloop<kHalves>(tmem_base + x * 128, desc_lo(q_smem + x * L::kTileBytes, 16),
+                              desc_lo(kv_smem + s * L::kTileBytes, 16), desc_hi_sw128(1024), idesc_qk);
         mma_commit(bar_sfull + 8 * x);
         return true;
       };
       // O_x += P_x V_j   (P_x read from TMEM where the softmax warps left it, over S_x)
-      auto issue_pv = [&](int x, int j) -> bool {
+      auto issue_pv = [&](int x, int j, bool wait_tile) -> bool {
         const int u = 2 * j + 1, s = u % kRing;
+        if (wait_tile && !mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
         if (!mbar_wait(bar_pfull + 8 * x, j & 1, abort_flag)) return false;
-        if (!mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t va = kv_smem + s * L::kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < kBN / 32; ++kk)
-          mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + kk * 8,
-                 smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
+        const uint32_t v_lo = desc_lo(kv_smem + s * L::kTileBytes, kHalfBytes);
+        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128, v_lo, desc_hi_sw128(1024), idesc_pv, j > 0 ? 1u : 0u);
         // the second half of P arrives while the first half is being multiplied
         if (!mbar_wait(bar_pfull_hi + 8 * x, j & 1, abort_flag)) return false;
         tc_fence_after();
-#pragma unroll
-        for (int kk = kBN / 32; kk < kBN / 16; ++kk)
-          mma_ts(tmem_base + 256 + x * 128, tmem_base + x * 128 + kk * 8,
-                 smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_pv, 1u);
+        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128 + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
         if (j == n_kv[x] - 1) mma_commit(bar_ofinal + 8 * x);
         return true;
       };
-      if (ok && n_kv[0] > 0) ok = issue_qk(0, 0);
-      if (ok && n_kv[1] > 0) ok = issue_qk(1, 0);
+      if (ok && n_kv[0] > 0) ok = issue_qk(0, 0, true);
+      if (ok && n_kv[1] > 0) ok = issue_qk(1, 0, n_kv[0] == 0);
       if (ok) mma_commit(bar_empty + 8 * 0);                   // K_0's buffer: free once both S tiles are done
       for (int j = 0; ok && j < n_kv_max; ++j) {
-        if (j < n_kv[0]) {
-          if (!(ok = issue_pv(0, j))) break;
-          if (j + 1 < n_kv[0] && !(ok = issue_qk(0, j + 1))) break;
+        const bool a_pv = j < n_kv[0], a_qk = j + 1 < n_kv[0];
+        if (a_pv) {
+          if (!(ok = issue_pv(0, j, true))) break;
+          if (a_qk && !(ok = issue_qk(0, j + 1, true))) break;
         }
         if (j < n_kv[1]) {
-          if (!(ok = issue_pv(1, j))) break;
+          if (!(ok = issue_pv(1, j, !a_pv))) break;
         }
         mma_commit(bar_empty + 8 * ((2 * j + 1) % kRing));     // V_j
-        if (j + 1 < n_kv[1] && !(ok = issue_qk(1, j + 1))) break;
+        if (j + 1 < n_kv[1] && !(ok = issue_qk(1, j + 1, !a_qk))) break;
         if (j + 1 < n_kv_max) mma_commit(bar_empty + 8 * ((2 * j + 2) % kRing));   // K_{j+1}
       }
     }

@@ -155,6 +155,59 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ---- batched issue: several tcgen05.mma from ONE asm statement ------------------------------------------
+// The issuing thread is a single lane, so every instruction it spends on descriptor arithmetic delays
+// the next MMA.  A descriptor's low word holds the (address >> 4); stepping along K only adds a small
+// constant to it, so a whole K-loop is emitted as add / mov.b64 / mma triples with immediates.
+//   lo word: (smem address >> 4) | (leading byte offset >> 4) << 16      hi word: see desc_hi_sw128()
+__host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);        // stride offset | version | 128B swizzle
+}
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+
+#define RELAXKV_MMA_SS_STEP(OFF, PRED)                                                         \
+  "add.u32 ta, %1, " #OFF ";\n\tadd.u32 tb, %2, " #OFF ";\n\t"                                    \
+  "mov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"                                           \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " #PRED ";\n\t"
+
+// D[tmem] = A[smem] * B[smem] over K = 64 * HALVES (both operands K-major, 128B swizzle, halves 16 KB apart
+// for A when a_half_step16 = 1024 and for B when the same): the first MMA overwrites D.
+template <int HALVES>
+__device__ __forceinline__ void mma_ss_kloop(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+  if (HALVES == 2) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        RELAXKV_MMA_SS_STEP(0, p0) RELAXKV_MMA_SS_STEP(2, p1) RELAXKV_MMA_SS_STEP(4, p1) RELAXKV_MMA_SS_STEP(6, p1)
+        RELAXKV_MMA_SS_STEP(1024, p1) RELAXKV_MMA_SS_STEP(1026, p1) RELAXKV_MMA_SS_STEP(1028, p1) RELAXKV_MMA_SS_STEP(1030, p1)
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        RELAXKV_MMA_SS_STEP(0, p0) RELAXKV_MMA_SS_STEP(2, p1) RELAXKV_MMA_SS_STEP(4, p1) RELAXKV_MMA_SS_STEP(6, p1)
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+  }
+}
+
+#define RELAXKV_MMA_TS_STEP(AOFF, BOFF, PRED)                                                  \
+  "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                                  \
+  "mov.b64 db, {tb, %3};\n\t"                                                                  \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %4, " #PRED ";\n\t"
+
+// D[tmem] (+)= A[tmem] * B[smem] for four K steps of 16: A advances 8 columns, B (MN-major, 128B swizzle)
+// 2048 bytes per step.  acc_first = 0 makes the first MMA overwrite D.
+__device__ __forceinline__ void mma_ts_4steps(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                              uint32_t acc_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      RELAXKV_MMA_TS_STEP(0, 0, p0) RELAXKV_MMA_TS_STEP(8, 128, p1) RELAXKV_MMA_TS_STEP(16, 256, p1) RELAXKV_MMA_TS_STEP(24, 384, p1)
+      "}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first) : "memory");
+}
+
 // ---- descriptors ------------------------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle, tiles whose 8-row groups are 1024 bytes apart.
 //   K-major operand  (rows of 64 bf16 = 128 B):       lbo ignored (1),  sbo = 1024
