@@ -258,6 +258,14 @@ relaxkv_status relaxkv_sparse_ctx_attention_simt(
     void* workspace, size_t workspace_bytes, relaxkv_stream stream);
 
 /*
+ * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on
+ * a barrier nothing will ever complete.  The wait gives up after its limit (0.4 s), the kernel ends
+ * normally and RELAXKV_ERR_TIMEOUT is recorded in the device status word - the same path a stuck
+ * pipeline takes in the attention and scoring kernels.  Nothing hangs or faults.
+ */
+relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream);
+
+/*
  * Synchronises `stream`, copies the device status word (a relaxkv_status: RELAXKV_OK,
  * RELAXKV_ERR_BAD_INDEX or RELAXKV_ERR_TIMEOUT, the first problem recorded wins) to
  * *h_status_out and clears it.  h_detail_out (NULL or host int32[4]) receives where it happened:

@@ -178,6 +178,54 @@ void relaxkv_oracle_mix_context(const uint16_t* cache_k, const uint16_t* cache_v
         }
 }
 
+/* ---- Appendix A.3 (controlled configurations): any target list against any context list ----
+ * The variants (global targets P, Global / Layerwise Sparse context sets U_l) keep the definition
+ * C_l(p) = X intersect {j <= p} with their own context list X and target list; a target need not be
+ * a member of X.  limit[rho] = (number of context positions <= tgt_pos[rho]) - 1, i.e. -1 when the
+ * target sees nothing.  Both lists ascending. */
+void relaxkv_oracle_limits(const int32_t* ctx_pos, int32_t n_ctx, const int32_t* tgt_pos, int32_t n_tgt, int32_t* limit) {
+    for (int32_t r = 0; r < n_tgt; ++r) {
+        int32_t n = 0;
+        for (int32_t c = 0; c < n_ctx; ++c) if (ctx_pos[c] <= tgt_pos[r]) ++n;
+        limit[r] = n - 1;
+    }
+}
+
+/* Mixed context for explicit lists (Section 3.4 equation with R_l := the target list):
+ * ctx[c] = new[rho] if ctx_pos[c] == tgt_pos[rho] for some rho, else cache[ctx_pos[c]]. */
+void relaxkv_oracle_mix_context_lists(const uint16_t* cache_k, const uint16_t* cache_v,
+                                      int64_t tok_stride, int64_t head_stride,
+                                      const uint16_t* k_new, const uint16_t* v_new,
+                                      const int32_t* ctx_pos, int32_t n_ctx, const int32_t* tgt_pos, int32_t n_tgt,
+                                      int Hkv, int D, uint16_t* ctx_k, uint16_t* ctx_v) {
+    for (int32_t c = 0; c < n_ctx; ++c) {
+        int32_t rho = -1;
+        if (k_new && v_new)
+            for (int32_t r = 0; r < n_tgt; ++r) if (tgt_pos[r] == ctx_pos[c]) rho = r;
+        for (int g = 0; g < Hkv; ++g) {
+            uint16_t* dk = ctx_k + ((int64_t)c * Hkv + g) * D;
+            uint16_t* dv = ctx_v + ((int64_t)c * Hkv + g) * D;
+            if (rho >= 0) {
+                memcpy(dk, k_new + ((int64_t)rho * Hkv + g) * D, sizeof(uint16_t) * D);
+                memcpy(dv, v_new + ((int64_t)rho * Hkv + g) * D, sizeof(uint16_t) * D);
+            } else {
+                const int64_t src = (int64_t)ctx_pos[c] * tok_stride + (int64_t)g * head_stride;
+                memcpy(dk, cache_k + src, sizeof(uint16_t) * D);
+                memcpy(dv, cache_v + src, sizeof(uint16_t) * D);
+            }
+        }
+    }
+}
+
+/* ---- Appendix B (global repair target sweep): g_i = (1/L) sum_l a_{l,i} ---- */
+void relaxkv_oracle_mean_scores(const double* scores, int L, int64_t T, double* g) {
+    for (int64_t i = 0; i < T; ++i) {
+        double a = 0.0;
+        for (int l = 0; l < L; ++l) a += scores[(int64_t)l * T + i];
+        g[i] = a / (double)L;
+    }
+}
+
 /* ---- Section 3.3 / Algorithm 1, sparse-context repair attention ----
  * For each listed target row rho (rows[] indexes q_new and limit[]), head h:
  *   O[rho,h,:] = sum_{c<=limit[rho]} softmax_c(scale*<q, ctx_k[c, h/G]>) * ctx_v[c, h/G, :]
@@ -194,6 +242,11 @@ void relaxkv_oracle_attention(const uint16_t* q_new, const uint16_t* ctx_k, cons
             const int32_t rho = rows[r];
             const int32_t cmax = limit[rho];
             const int g = h / G;
+            if (cmax < 0) {            /* empty context (only possible with explicit lists): defined as zero output */
+                for (int d = 0; d < D; ++d) out[((int64_t)r * H + h) * D + d] = 0.0;
+                if (lse) lse[(int64_t)r * H + h] = -INFINITY;
+                continue;
+            }
             const uint16_t* qr = q_new + ((int64_t)rho * H + h) * D;
             double m = -INFINITY;
             for (int32_t c = 0; c <= cmax; ++c) {

@@ -226,6 +226,51 @@ def repair_attention(cache_k, cache_v, q_new, k_new, v_new, u_pos, r_rank, scale
     return attention(q_new, ck, cv, limit, scale, rows)
 
 
+def limits(ctx_pos, tgt_pos) -> np.ndarray:
+    """Causal limit of each target in an arbitrary context list: index of the last context position
+    <= the target's position, -1 if there is none (Appendix A.3: C_l(p) = X intersect {j <= p})."""
+    lib = _load()
+    ctx_pos, tgt_pos = _i32(ctx_pos), _i32(tgt_pos)
+    out = np.empty(tgt_pos.shape[0], dtype=np.int32)
+    lib.relaxkv_oracle_limits(_p(ctx_pos), ctx_pos.shape[0], _p(tgt_pos), tgt_pos.shape[0], _p(out))
+    return out
+
+
+def mix_context_lists(cache_k, cache_v, k_new, v_new, ctx_pos, tgt_pos):
+    """Mixed fresh/cached K/V over an explicit context list for an explicit target list."""
+    lib = _load()
+    T, Hkv, D = cache_k.shape
+    ts, hs = _kv_strides(cache_k)
+    assert _kv_strides(cache_v) == (ts, hs)
+    ctx_pos, tgt_pos = _i32(ctx_pos), _i32(tgt_pos)
+    ck = np.empty((ctx_pos.shape[0], Hkv, D), dtype=np.uint16)
+    cv = np.empty_like(ck)
+    kn = None if k_new is None else _u16(k_new)
+    vn = None if v_new is None else _u16(v_new)
+    lib.relaxkv_oracle_mix_context_lists(_p(cache_k), _p(cache_v), ctypes.c_int64(ts), ctypes.c_int64(hs), _p(kn), _p(vn),
+                                         _p(ctx_pos), ctx_pos.shape[0], _p(tgt_pos), tgt_pos.shape[0], Hkv, D,
+                                         _p(ck), _p(cv))
+    return ck, cv
+
+
+def list_attention(cache_k, cache_v, q_new, k_new, v_new, ctx_pos, tgt_pos, scale, rows=None):
+    """Repair attention of the controlled configurations (Appendix A.3): targets tgt_pos (any ascending
+    list) attend to the context list ctx_pos under C(p) = ctx intersect {j <= p}; context entries that
+    are targets contribute their fresh K/V.  A target with an empty context yields zeros (lse = -inf)."""
+    ck, cv = mix_context_lists(cache_k, cache_v, k_new, v_new, ctx_pos, tgt_pos)
+    return attention(q_new, ck, cv, limits(ctx_pos, tgt_pos), scale, rows)
+
+
+def mean_scores(scores: np.ndarray) -> np.ndarray:
+    """g_i = mean over layers of a_{l,i} (Appendix B, global repair target sweep)."""
+    lib = _load()
+    scores = np.ascontiguousarray(scores, dtype=np.float64)
+    L, T = scores.shape
+    g = np.empty(T, dtype=np.float64)
+    lib.relaxkv_oracle_mean_scores(_p(scores), L, ctypes.c_int64(T), _p(g))
+    return g
+
+
 def scatter(cache_k, cache_v, k_new, v_new, positions) -> None:
     """Cache update in place on the numpy arrays (Section 3.4)."""
     lib = _load()

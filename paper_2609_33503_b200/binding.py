@@ -23,7 +23,7 @@ ENTRY_POINTS = (
     "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
-    "relaxkv_build_active_sets_static",
+    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
 )
 
 
@@ -237,6 +237,11 @@ def relaxkv_gather_kv(shape: Shape, mode: int, cache: CacheView, k_new: Optional
                                    _ptr(u_cu), _ptr(r_rank), _ptr(r_cu_layer), _i32(max_ctx), _ptr(k_ctx_out),
                                    _ptr(v_ctx_out), ctypes.c_int64(k_ctx_out.shape[0]), _stream(stream)),
            "relaxkv_gather_kv")
+
+
+def relaxkv_debug_wait_timeout(stream=None) -> None:
+    """Launches the bounded-wait probe: ends after ~0.4 s with RELAXKV_ERR_TIMEOUT in the status word."""
+    _check(lib().relaxkv_debug_wait_timeout(_stream(stream)), "relaxkv_debug_wait_timeout")
 
 
 def relaxkv_read_device_status(stream=None):

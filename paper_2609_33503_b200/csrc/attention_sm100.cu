@@ -363,6 +363,21 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   }
 }
 
+// Test utility: one thread waits (bounded) on an mbarrier that nothing ever completes.  Exercises the
+// give-up path of every kernel's waits without hanging anything: the wait expires after the limit,
+// the abort flag is raised and RELAXKV_ERR_TIMEOUT lands in the device status word.
+__global__ void wait_timeout_probe_kernel(DeviceStatus* st) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ volatile int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_barrier_init();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag);
+    if (!ok && abort_flag) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, -1, -1);
+  }
+}
+
 // ---- host side ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -443,4 +458,11 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention(
   if (shape->head_dim == 128)
     return launch_attention<128>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
   return launch_attention<64>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
+}
+
+extern "C" relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream) {
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st);
+  return launch_ok();
 }

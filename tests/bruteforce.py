@@ -73,8 +73,12 @@ def attention(cache_k, cache_v, q_new, k_new, v_new, U, R_pos, scale, full_prefi
         s = (q[:, h, :] @ k_eff[:, h // G, :].T) * scale                      # [n_r, T]
         s = np.where(vis, s, -np.inf)
         m = s.max(axis=1, keepdims=True)
+        empty = ~np.isfinite(m[:, 0])                                         # no visible position at all
+        m = np.where(np.isfinite(m), m, 0.0)
         p = np.exp(s - m)
         z = p.sum(axis=1, keepdims=True)
-        out[:, h, :] = (p / z) @ v_eff[:, h // G, :]
-        lse[:, h] = (m + np.log(z))[:, 0]
+        z_safe = np.where(z > 0, z, 1.0)
+        out[:, h, :] = (p / z_safe) @ v_eff[:, h // G, :]
+        with np.errstate(divide="ignore"):
+            lse[:, h] = np.where(empty, -np.inf, (m + np.log(z_safe))[:, 0])
     return out, lse, int(vis.sum())

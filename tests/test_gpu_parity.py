@@ -331,3 +331,19 @@ def test_bad_index_lists_are_reported_not_faulted():
     s.scatter(0, B().CacheView(k2, v2, [0]), f.k_new, f.v_new, case.max_targets(0))
     st, _ = B().relaxkv_read_device_status()
     assert st == B().ERR_BAD_INDEX
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable():
+    """A wait that can never be satisfied gives up after its limit: the kernel returns, the status word
+    says RELAXKV_ERR_TIMEOUT, and the next call on the same context works."""
+    import time
+    t0 = time.time()
+    B().relaxkv_debug_wait_timeout()
+    st, detail = B().relaxkv_read_device_status()
+    assert st == B().ERR_TIMEOUT, (st, detail)
+    assert 0.2 < time.time() - t0 < 5.0
+    case = Case(inputs.tiny())
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    out, lse = run_attention(case, s, 0, B().CTX_UNION, simt=False)
+    check_attention(case, 0, out, lse, False)

@@ -265,6 +265,48 @@ def test_attention_special_cases():
     np.testing.assert_array_equal(mv[ranks], vn)
 
 
+# ------------------------------------------ controlled configurations (explicit lists) ----
+
+def test_list_attention_reduces_to_the_method_and_matches_bruteforce():
+    rng = np.random.default_rng(21)
+    H, Hkv, D, T, L, k = 4, 2, 16, 57, 3, 10
+    ck, cv = rand_bits(rng, T, Hkv, D), rand_bits(rng, T, Hkv, D)
+    anchors = np.stack([np.sort(rng.choice(T, size=k, replace=False)) for _ in range(L)]).astype(np.int32)
+    s = orc.active_sets(anchors, T)
+    scale = 0.25
+    l = 1
+    pos = s.positions(l)
+    qn, kn, vn = rand_bits(rng, len(pos), H, D), rand_bits(rng, len(pos), Hkv, D), rand_bits(rng, len(pos), Hkv, D)
+    # context = U, targets = R_l  ->  the method itself; context = everything -> the full-prefix control
+    a, la = orc.list_attention(ck, cv, qn, kn, vn, s.u_pos, pos, scale)
+    b, lb = orc.repair_attention(ck, cv, qn, kn, vn, s.u_pos, s.ranks(l), scale)
+    np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(orc.limits(s.u_pos, pos), s.ranks(l))
+    c, _ = orc.list_attention(ck, cv, qn, kn, vn, np.arange(T), pos, scale)
+    d, _ = orc.repair_attention(ck, cv, qn, kn, vn, s.u_pos, s.ranks(l), scale, full_prefix=True)
+    np.testing.assert_array_equal(c, d)
+    # arbitrary targets that need not lie in the context list (global targets, sparse context variants)
+    for trial in range(4):
+        ctx = np.sort(rng.choice(np.arange(3, T), size=15, replace=False)).astype(np.int32)
+        tgt = np.sort(rng.choice(T, size=12, replace=False)).astype(np.int32)
+        tgt[0] = 1                                   # before every context position: empty context
+        tgt = np.unique(tgt)
+        q2, k2, v2 = rand_bits(rng, len(tgt), H, D), rand_bits(rng, len(tgt), Hkv, D), rand_bits(rng, len(tgt), Hkv, D)
+        out, lse = orc.list_attention(ck, cv, q2, k2, v2, ctx, tgt, scale)
+        ref, ref_lse, _ = bf.attention(ck, cv, q2, k2, v2, ctx, tgt, scale)
+        np.testing.assert_allclose(out, ref, rtol=1e-10, atol=1e-12)
+        assert np.all(out[0] == 0) and np.all(np.isneginf(lse[0]))          # the reading for an empty context
+        np.testing.assert_allclose(lse[1:], ref_lse[1:], rtol=1e-12)
+        lim = orc.limits(ctx, tgt)
+        assert lim[0] == -1 and all(lim[i] == np.searchsorted(ctx, tgt[i], side="right") - 1 for i in range(len(tgt)))
+
+
+def test_mean_scores():
+    rng = np.random.default_rng(22)
+    a = rng.random((5, 33))
+    np.testing.assert_allclose(orc.mean_scores(a), a.mean(axis=0), rtol=1e-15)
+
+
 # ------------------------------------------------------------------ update ----
 
 def test_scatter_semantics_and_order_equivalence():
