@@ -246,6 +246,38 @@ relaxkv_status relaxkv_gather_kv(
     relaxkv_stream stream);
 
 /*
+ * Repair attention for explicit target and context lists - the paper's controlled configurations
+ * (Appendix A.3, table of configurations; Section 4.4 ablation; Appendix B): global repair targets P
+ * with context C(p) = U intersect {j <= p} (RelaxKV^G, global target sweep), Global Sparse and Layerwise
+ * Sparse context sets U_l with the method's targets R_l.  For request b the targets are the positions
+ * tgt_pos[tgt_cu[b] .. tgt_cu[b+1]) and the context list is ctx_pos[ctx_cu[b] .. ctx_cu[b+1]), both
+ * ascending; tgt_cu[0] must be 0.  Target rho at position p attends to the context entries with
+ * position <= p; an entry whose position is itself a target contributes that target's fresh K/V, every
+ * other entry the cached K/V (Section 3.4 equation with R_l := the target list).  A target need not be a
+ * context entry (then it does not see itself); a target with no visible entry gets a zero output row and
+ * lse = -inf (the paper does not define that case).  With ctx = U, tgt = R_l this equals
+ * relaxkv_sparse_ctx_attention; with ctx = all positions, its full-prefix mode.
+ * q_new/k_new/v_new/out rows follow the packed target order; other arguments as above.
+ */
+relaxkv_status relaxkv_list_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache,
+    const void* q_new, const void* k_new, const void* v_new,
+    const int32_t* ctx_pos, const int32_t* ctx_cu, const int32_t* tgt_pos, const int32_t* tgt_cu,
+    int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
+    void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/* Cache update for an explicit target list (Section 3.4): cache entries at tgt_pos receive k_new / v_new. */
+relaxkv_status relaxkv_scatter_kv_lists(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* k_new, const void* v_new,
+    const int32_t* tgt_pos, const int32_t* tgt_cu, const int32_t* h_max_targets, relaxkv_stream stream);
+
+/* Across-layer mean score g_i = (1/L) sum_l a_{l,i} (Appendix B; also the Global Sparse context source):
+ * scores device fp32 [n_layers, sum_b T_c] -> mean_out device fp32 [sum_b T_c], summed in layer order.
+ * Feed mean_out to relaxkv_select_topk (n_layers = 1) for the global target set or the shared context set. */
+relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers, const float* scores,
+                                   float* mean_out, relaxkv_stream stream);
+
+/*
  * Test utility: the same result as relaxkv_sparse_ctx_attention from a plain SIMT kernel (one warp
  * per output row, fp32 throughout, no tensor cores).  A second opinion for debugging; far slower.
  */

@@ -23,7 +23,8 @@ ENTRY_POINTS = (
     "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
-    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
+    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_list_attention",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores",
 )
 
 
@@ -237,6 +238,29 @@ def relaxkv_gather_kv(shape: Shape, mode: int, cache: CacheView, k_new: Optional
                                    _ptr(u_cu), _ptr(r_rank), _ptr(r_cu_layer), _i32(max_ctx), _ptr(k_ctx_out),
                                    _ptr(v_ctx_out), ctypes.c_int64(k_ctx_out.shape[0]), _stream(stream)),
            "relaxkv_gather_kv")
+
+
+def relaxkv_list_attention(shape: Shape, cache: CacheView, q_new: torch.Tensor, k_new: Optional[torch.Tensor],
+                           v_new: Optional[torch.Tensor], ctx_pos: torch.Tensor, ctx_cu: torch.Tensor,
+                           tgt_pos: torch.Tensor, tgt_cu: torch.Tensor, max_targets: Sequence[int],
+                           max_ctx: Sequence[int], out: torch.Tensor, workspace: torch.Tensor,
+                           lse_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(lib().relaxkv_list_attention(shape.ref(), cache.ref(), _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(ctx_pos),
+                                        _ptr(ctx_cu), _ptr(tgt_pos), _ptr(tgt_cu), ctypes.c_int64(q_new.shape[0]),
+                                        _i32(max_targets), _i32(max_ctx), _ptr(out), _ptr(lse_out), _ptr(workspace),
+                                        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)),
+           "relaxkv_list_attention")
+
+
+def relaxkv_scatter_kv_lists(shape: Shape, cache: CacheView, k_new: torch.Tensor, v_new: torch.Tensor,
+                             tgt_pos: torch.Tensor, tgt_cu: torch.Tensor, max_targets: Sequence[int], stream=None) -> None:
+    _check(lib().relaxkv_scatter_kv_lists(shape.ref(), cache.ref(), _ptr(k_new), _ptr(v_new), _ptr(tgt_pos), _ptr(tgt_cu),
+                                          _i32(max_targets), _stream(stream)), "relaxkv_scatter_kv_lists")
+
+
+def relaxkv_mean_scores(shape: Shape, n_layers: int, scores: torch.Tensor, mean_out: torch.Tensor, stream=None) -> None:
+    _check(lib().relaxkv_mean_scores(shape.ref(), int(n_layers), _ptr(scores), _ptr(mean_out), _stream(stream)),
+           "relaxkv_mean_scores")
 
 
 def relaxkv_debug_wait_timeout(stream=None) -> None:

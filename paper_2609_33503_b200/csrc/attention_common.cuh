@@ -20,7 +20,8 @@ inline relaxkv_status prepare_attention(
     const void* q_new, const void* k_new, const void* v_new,
     const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
     int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
-    void* out, void* workspace, size_t workspace_bytes, cudaStream_t stream, AttnPlan& plan) {
+    void* out, void* workspace, size_t workspace_bytes, cudaStream_t stream, AttnPlan& plan,
+    const int32_t* fresh_row = nullptr) {
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if ((rc = check_cache(shape, cache, true)) != RELAXKV_OK) return rc;
@@ -52,8 +53,8 @@ inline relaxkv_status prepare_attention(
   plan.kctx = reinterpret_cast<uint16_t*>(base + ws.kctx);
   plan.vctx = reinterpret_cast<uint16_t*>(base + ws.vctx);
   plan.ctx_rows = ws.ctx_rows_cap;
-  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, need_ctx + kCtxPadRows,
-                       plan.kctx, plan.vctx, plan.ctx_rows, stream);
+  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, fresh_row,
+                       need_ctx + kCtxPadRows, plan.kctx, plan.vctx, plan.ctx_rows, stream);
 }
 
 }  // namespace relaxkv

@@ -46,7 +46,7 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
-                       int mode, int H, int Hkv, int tile_targets, float scale_log2,
+                       int mode, int allow_empty, int H, int Hkv, int tile_targets, float scale_log2,
                        const int* __restrict__ u_pos, const int* __restrict__ u_cu,
                        const int* __restrict__ r_rank, const int* __restrict__ r_cu,
                        long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
@@ -224,9 +224,12 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const bool row_valid = (row < tile_targets * G) && (t_local < n_valid[x]);
     const int rho_t = rho0 + x * tile_targets + t_local;
     int limit = 0;
+    bool row_empty = false;                                     // explicit lists: a target that sees no context entry
     if (row_valid) {
       const int c = r_rank[r_cu[b] + rho_t];
-      if (c < 0 || c >= nu) {
+      if (c == -1 && allow_empty) {
+        row_empty = true;
+      } else if (c < 0 || c >= nu) {
         report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
       } else {
         limit = (mode == RELAXKV_CTX_UNION) ? c : u_pos[u_cu[b] + c];
@@ -321,7 +324,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     if (ok && my_n > 0) {
       tc_fence_after();
-      const float inv = 1.f / z;
+      const float inv = row_empty ? 0.f : 1.f / z;              // an empty context is defined as a zero output row
       const long long orow = q_row_base + x * tile_targets + t_local;
       uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
 #pragma unroll
@@ -343,7 +346,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
         }
       }
-      if (row_valid && lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = (m + log2f(z)) * kLn2A;
+      if (row_valid && lse_out)
+        lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = row_empty ? -INFINITY : (m + log2f(z)) * kLn2A;
     }
   }
 
@@ -360,6 +364,43 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Explicit lists (the paper's controlled configurations): per target the index of the last context entry
+// at or before its position (-1: none), per context entry the row of the fresh K/V that replaces it (-1:
+// cached).  rt.tile_cu = prefix of the host bounds on the target counts, rt.bound_b = bounds on the context.
+__global__ void build_list_maps_kernel(ReqTable rt, const int* __restrict__ ctx_pos, const int* __restrict__ ctx_cu,
+                                       const int* __restrict__ tgt_pos, const int* __restrict__ tgt_cu,
+                                       long long ctx_bound_total, int* __restrict__ limit, int* __restrict__ fresh_row,
+                                       DeviceStatus* st) {
+  const int B = rt.n_req;
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long n_tgt_slots = rt.tile_cu[B];
+  if (i < n_tgt_slots) {
+    const int b = find_segment(rt.tile_cu, B, (int)i);
+    const int rho = (int)i - rt.tile_cu[b];
+    const int t0 = tgt_cu[b], nt = tgt_cu[b + 1] - t0;
+    if (rho == 0 && (nt > rt.bound_a[b] || tgt_cu[0] != 0)) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nt, tgt_cu[0]);
+    if (rho < nt) {
+      const int p = tgt_pos[t0 + rho];
+      const int c0 = ctx_cu[b], nc = ctx_cu[b + 1] - c0;
+      int lo = 0, hi = nc;                                   // first context entry with position > p
+      while (lo < hi) { const int mid = (lo + hi) >> 1; if (ctx_pos[c0 + mid] <= p) lo = mid + 1; else hi = mid; }
+      if (p < 0 || p >= rt.ctx_len[b]) { report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, p, rt.ctx_len[b]); lo = 1; }
+      limit[t0 + rho] = lo - 1;
+    }
+  } else if (i < n_tgt_slots + ctx_bound_total) {
+    const long long x = i - n_tgt_slots;
+    if (x < ctx_cu[B]) {
+      int b = 0;
+      while (b + 1 < B && x >= ctx_cu[b + 1]) ++b;
+      const int p = ctx_pos[x];
+      const int t0 = tgt_cu[b], nt = tgt_cu[b + 1] - t0;
+      int lo = 0, hi = nt;
+      while (lo < hi) { const int mid = (lo + hi) >> 1; if (tgt_pos[t0 + mid] < p) lo = mid + 1; else hi = mid; }
+      fresh_row[x] = (lo < nt && tgt_pos[t0 + lo] == p) ? (t0 + lo) : -1;
+    }
   }
 }
 
@@ -413,7 +454,7 @@ template <int D>
 static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, AttnPlan& plan, const void* q_new,
                                        const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank,
                                        const int32_t* r_cu_layer, long long n_target_rows, void* out, float* lse_out,
-                                       cudaStream_t stream) {
+                                       cudaStream_t stream, int allow_empty = 0) {
   const int H = shape->n_q_heads, Hkv = shape->n_kv_heads, G = H / Hkv;
   const int tile_targets = kBM / G;
   const int B = shape->n_req;
@@ -434,7 +475,7 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess)
     return RELAXKV_ERR_CUDA;
   kern<<<(unsigned)grid, kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
-      tm_q, tm_k, tm_v, plan.rt, mode, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
+      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
       r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, st);
   return launch_ok();
 }
@@ -465,4 +506,55 @@ extern "C" relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream) {
   if (!st) return RELAXKV_ERR_CUDA;
   wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st);
   return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_list_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache,
+    const void* q_new, const void* k_new, const void* v_new,
+    const int32_t* ctx_pos, const int32_t* ctx_cu, const int32_t* tgt_pos, const int32_t* tgt_cu,
+    int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
+    void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (!ctx_pos || !ctx_cu || !tgt_pos || !tgt_cu || !h_max_targets || !h_max_ctx || !workspace)
+    return RELAXKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return RELAXKV_ERR_INVALID_ARG;
+  const WsLayout ws = ws_layout(shape, 1);
+  if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
+  int* limit = reinterpret_cast<int*>(static_cast<char*>(workspace) + ws.list_limit);
+  int* fresh = reinterpret_cast<int*>(static_cast<char*>(workspace) + ws.list_fresh);
+  // 1. the two maps
+  ReqTable rt;
+  fill_req_table(rt, shape, nullptr, nullptr);
+  long long tgt_total = 0, ctx_total = 0;
+  for (int b = 0; b < shape->n_req; ++b) {
+    if (h_max_targets[b] < 0 || h_max_targets[b] > shape->h_ctx_len[b] || h_max_ctx[b] < 0 ||
+        h_max_ctx[b] > shape->h_ctx_len[b])
+      return RELAXKV_ERR_INVALID_ARG;
+    rt.bound_a[b] = h_max_targets[b];
+    rt.bound_b[b] = h_max_ctx[b];
+    tgt_total += h_max_targets[b];
+    ctx_total += h_max_ctx[b];
+    rt.tile_cu[b + 1] = (int)tgt_total;
+  }
+  if (tgt_total + ctx_total > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  if (tgt_total + ctx_total > 0) {
+    const long long n = tgt_total + ctx_total;
+    build_list_maps_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(rt, ctx_pos, ctx_cu, tgt_pos, tgt_cu, ctx_total,
+                                                                          limit, fresh, st);
+    if ((rc = launch_ok()) != RELAXKV_OK) return rc;
+  }
+  // 2. gather (fresh rows resolved through the map) and 3. the attention kernel with the limits as "ranks"
+  AttnPlan plan;
+  rc = prepare_attention(shape, RELAXKV_CTX_UNION, cache, q_new, k_new, v_new, ctx_pos, ctx_cu, limit, tgt_cu, n_target_rows,
+                         h_max_targets, h_max_ctx, out, workspace, workspace_bytes, stream, plan, fresh);
+  if (rc != RELAXKV_OK) return rc;
+  if (shape->head_dim == 128)
+    return launch_attention<128>(shape, RELAXKV_CTX_UNION, plan, q_new, ctx_pos, ctx_cu, limit, tgt_cu, n_target_rows, out,
+                                 lse_out, stream, 1);
+  return launch_attention<64>(shape, RELAXKV_CTX_UNION, plan, q_new, ctx_pos, ctx_cu, limit, tgt_cu, n_target_rows, out,
+                              lse_out, stream, 1);
 }

@@ -118,6 +118,8 @@ inline int score_blocks(int q_len, int group) {
 struct WsLayout {
   // attention: materialised mixed context K~ / V~  [ctx_rows_cap, H_kv, D] bf16
   size_t kctx, vctx; long long ctx_rows_cap;
+  // explicit-list attention: limit [sumT] i32 | fresh_row [sumT] i32
+  size_t list_limit, list_fresh;
   // scoring: lse [H, sumQ] f32 | part [2*kScoreSplitsMax, H, sumQ] float2 | colpart [2*H_kv*max_blocks, sumT] f32
   size_t lse, part, colpart;
   // sets: counts [B + L*B] i32
@@ -134,6 +136,8 @@ inline WsLayout ws_layout(const relaxkv_shape* s, int n_layers) {
   size_t a = 0;
   w.kctx = a; a = align_up(a + (size_t)w.ctx_rows_cap * row_bytes, 1024);
   w.vctx = a; a = align_up(a + (size_t)w.ctx_rows_cap * row_bytes, 1024);
+  w.list_limit = a; a = align_up(a + (size_t)sum_t * 4, 256);
+  w.list_fresh = a; a = align_up(a + (size_t)sum_t * 4, 256);
   size_t attn_total = a;
   a = 0;
   w.lse = a; a = align_up(a + (size_t)s->n_q_heads * sum_q * 4, 256);

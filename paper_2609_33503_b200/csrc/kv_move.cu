@@ -36,7 +36,7 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
                   long long tok_stride, long long head_stride,
                   const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                   const int* __restrict__ u_pos, const int* __restrict__ u_cu,
-                  const int* __restrict__ r_rank, const int* __restrict__ r_cu,
+                  const int* __restrict__ r_rank, const int* __restrict__ r_cu, const int* __restrict__ fresh_row,
                   uint16_t* __restrict__ k_out, uint16_t* __restrict__ v_out, long long ctx_rows,
                   DeviceStatus* st) {
   __shared__ long long src_off[kGatherRows];   // element offset of the source row (head 0)
@@ -71,7 +71,11 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
         } else {
           kind = 0;
           off = (rt.tok_off[b] + p) * tok_stride;
-          if (k_new != nullptr && c >= 0) {
+          if (k_new != nullptr && fresh_row != nullptr) {
+            // explicit lists: the row of k_new that replaces this context entry was resolved beforehand
+            const int fr = __ldg(fresh_row + x);
+            if (fr >= 0) { kind = 1; off = (long long)fr * n_kv_heads * head_dim; }
+          } else if (k_new != nullptr && c >= 0) {
             const int rb = __ldg(r_cu + b), nr = __ldg(r_cu + b + 1) - rb;
             const int rho = warp_lower_bound(r_rank + rb, nr, c, lane);
             if (rho < nr && __ldg(r_rank + rb + rho) == c) {
@@ -135,7 +139,8 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
                   long long tok_stride, long long head_stride,
                   const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                   const int* __restrict__ u_pos, const int* __restrict__ u_cu,
-                  const int* __restrict__ r_rank, const int* __restrict__ r_cu, DeviceStatus* st) {
+                  const int* __restrict__ r_rank, const int* __restrict__ r_cu, int direct, DeviceStatus* st) {
+  // direct != 0: u_pos holds the targets' positions themselves (packed by r_cu); r_rank is not read
   __shared__ long long dst_off[kScatterRows];
   __shared__ long long src_off[kScatterRows];
   const int B = rt.n_req;
@@ -150,10 +155,14 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
       const int nr = r_cu[b + 1] - r_cu[b];
       if (rho == 0 && nr > rt.bound_a[b]) report(st, RELAXKV_ERR_BAD_INDEX, KID_SCATTER, b, nr);
       if (rho < nr) {
-        const int c = r_rank[r_cu[b] + rho];
-        const int nu = u_cu[b + 1] - u_cu[b];
-        int p = -1;
-        if (c >= 0 && c < nu) p = u_pos[u_cu[b] + c];
+        int c = -1, p = -1;
+        if (direct) {
+          p = u_pos[r_cu[b] + rho];
+        } else {
+          c = r_rank[r_cu[b] + rho];
+          const int nu = u_cu[b + 1] - u_cu[b];
+          if (c >= 0 && c < nu) p = u_pos[u_cu[b] + c];
+        }
         if (p < 0 || p >= rt.ctx_len[b]) {
           report(st, RELAXKV_ERR_BAD_INDEX, KID_SCATTER, c, p);
         } else {
@@ -186,8 +195,8 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
 
 relaxkv_status launch_gather(const relaxkv_shape* shape, int mode, const relaxkv_cache_view* cache,
                              const void* k_new, const void* v_new, const int32_t* u_pos, const int32_t* u_cu,
-                             const int32_t* r_rank, const int32_t* r_cu_layer, long long rows_to_cover,
-                             void* k_out, void* v_out, long long ctx_rows, cudaStream_t stream) {
+                             const int32_t* r_rank, const int32_t* r_cu_layer, const int32_t* fresh_row,
+                             long long rows_to_cover, void* k_out, void* v_out, long long ctx_rows, cudaStream_t stream) {
   ReqTable rt;
   fill_req_table(rt, shape, cache, nullptr);
   DeviceStatus* st = status_word();
@@ -200,7 +209,7 @@ relaxkv_status launch_gather(const relaxkv_shape* shape, int mode, const relaxkv
       static_cast<const uint16_t*>(cache->k), static_cast<const uint16_t*>(cache->v),
       cache->token_stride, cache->head_stride,
       static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new),
-      u_pos, u_cu, r_rank, r_cu_layer, static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out), ctx_rows, st);
+      u_pos, u_cu, r_rank, r_cu_layer, fresh_row, static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out), ctx_rows, st);
   return launch_ok();
 }
 
@@ -235,7 +244,7 @@ extern "C" relaxkv_status relaxkv_gather_kv(
     }
   }
   if (ctx_rows < need) return RELAXKV_ERR_INVALID_ARG;
-  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, need + kCtxPadRows,
+  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, nullptr, need + kCtxPadRows,
                        k_ctx_out, v_ctx_out, ctx_rows, static_cast<cudaStream_t>(stream));
 }
 
@@ -265,6 +274,35 @@ extern "C" relaxkv_status relaxkv_scatter_kv(
   scatter_kv_kernel<<<(unsigned)blocks, kScatterThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       rt, shape->n_kv_heads, shape->head_dim, static_cast<uint16_t*>(cache->k), static_cast<uint16_t*>(cache->v),
       cache->token_stride, cache->head_stride, static_cast<const uint16_t*>(k_new),
-      static_cast<const uint16_t*>(v_new), u_pos, u_cu, r_rank, r_cu_layer, st);
+      static_cast<const uint16_t*>(v_new), u_pos, u_cu, r_rank, r_cu_layer, 0, st);
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_scatter_kv_lists(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* k_new, const void* v_new,
+    const int32_t* tgt_pos, const int32_t* tgt_cu, const int32_t* h_max_targets, relaxkv_stream stream) {
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if ((rc = check_cache(shape, cache, true)) != RELAXKV_OK) return rc;
+  if (!tgt_pos || !tgt_cu || !k_new || !v_new || !aligned16(k_new) || !aligned16(v_new) || !h_max_targets)
+    return RELAXKV_ERR_INVALID_ARG;
+  ReqTable rt;
+  fill_req_table(rt, shape, cache, nullptr);
+  long long total = 0;
+  for (int b = 0; b < shape->n_req; ++b) {
+    if (h_max_targets[b] < 0) return RELAXKV_ERR_INVALID_ARG;
+    rt.bound_a[b] = h_max_targets[b];
+    total += h_max_targets[b];
+    if (total > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+    rt.tile_cu[b + 1] = (int)total;
+  }
+  if (total == 0) return RELAXKV_OK;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  const long long blocks = (total + kScatterRows - 1) / kScatterRows;
+  scatter_kv_kernel<<<(unsigned)blocks, kScatterThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      rt, shape->n_kv_heads, shape->head_dim, static_cast<uint16_t*>(cache->k), static_cast<uint16_t*>(cache->v),
+      cache->token_stride, cache->head_stride, static_cast<const uint16_t*>(k_new),
+      static_cast<const uint16_t*>(v_new), tgt_pos, tgt_cu, tgt_pos, tgt_cu, 1, st);
   return launch_ok();
 }

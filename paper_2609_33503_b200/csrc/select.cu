@@ -127,6 +127,15 @@ select_topk_kernel(ReqTable rt, int n_layers, const float* __restrict__ raw, flo
   }
 }
 
+// g[i] = (1/L) * sum over layers (in layer order) of scores[l, i]   (Appendix B, global repair target sweep)
+__global__ void mean_scores_kernel(int n_layers, long long sum_t, const float* __restrict__ scores, float* __restrict__ g) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= sum_t) return;
+  float a = 0.f;
+  for (int l = 0; l < n_layers; ++l) a += scores[(long long)l * sum_t + i];
+  g[i] = a / (float)n_layers;
+}
+
 relaxkv_status launch_select(const ReqTable& rt, int n_layers, const float* raw, float* norm, int* anchors,
                              cudaStream_t stream) {
   DeviceStatus* st = status_word();
@@ -150,4 +159,15 @@ extern "C" relaxkv_status relaxkv_select_topk(const relaxkv_shape* shape, int32_
   ReqTable rt;
   fill_req_table(rt, shape, nullptr, h_k);
   return launch_select(rt, n_layers, raw_scores, norm_scores_out, anchors_out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers, const float* scores,
+                                              float* mean_out, relaxkv_stream stream) {
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (n_layers < 1 || !scores || !mean_out) return RELAXKV_ERR_INVALID_ARG;
+  long long sum_t = 0;
+  for (int b = 0; b < shape->n_req; ++b) sum_t += shape->h_ctx_len[b];
+  mean_scores_kernel<<<(unsigned)((sum_t + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(n_layers, sum_t, scores, mean_out);
+  return launch_ok();
 }

@@ -347,3 +347,122 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
     s.build_active_sets(case.anchors_tensor())
     out, lse = run_attention(case, s, 0, B().CTX_UNION, simt=False)
     check_attention(case, 0, out, lse, False)
+
+
+# ------------------------------------------------ controlled configurations (explicit lists) ----
+
+def _pack(lists, device):
+    cu = np.concatenate([[0], np.cumsum([len(x) for x in lists])]).astype(np.int32)
+    flat = np.concatenate(lists).astype(np.int32) if sum(len(x) for x in lists) else np.zeros(0, np.int32)
+    return torch.from_numpy(flat).to(device), torch.from_numpy(cu).to(device), cu
+
+
+def _run_lists(case, s, l, ctx_lists, tgt_lists, fresh=None):
+    """GPU list attention for per-request context / target position lists; returns out, lse, fresh tensors."""
+    w = case.w
+    ctx_pos, ctx_cu, _ = _pack(ctx_lists, case.device)
+    tgt_pos, tgt_cu, tcu = _pack(tgt_lists, case.device)
+    if fresh is None:
+        qs, ks, vs = [], [], []
+        for b in range(w.n_req):
+            lo, hi = int(case.ctx_cu[b]), int(case.ctx_cu[b + 1])
+            q, k, v = inputs.fresh_qkv(w, l, b, case.k_cache[l][lo:hi], case.v_cache[l][lo:hi],
+                                       torch.from_numpy(np.asarray(tgt_lists[b], dtype=np.int64)))
+            qs.append(q); ks.append(k); vs.append(v)
+        fresh = (torch.cat(qs).contiguous(), torch.cat(ks).contiguous(), torch.cat(vs).contiguous())
+    q_new, k_new, v_new = fresh
+    out = torch.full_like(q_new, 3.0)
+    lse = torch.zeros(w.n_q_heads, q_new.shape[0], dtype=torch.float32, device=case.device)
+    B().relaxkv_list_attention(s.shape, case.cache_views()[l], q_new, k_new, v_new, ctx_pos, ctx_cu, tgt_pos, tgt_cu,
+                               [len(x) for x in tgt_lists], [len(x) for x in ctx_lists], out, s.workspace, lse_out=lse)
+    assert_status_ok()
+    return out, lse, fresh, tcu
+
+
+def test_list_attention_reduces_to_the_method(case):
+    """Context = U and targets = R_l through the explicit-list call give the method's own output bits."""
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    l = case.w.n_layers - 1
+    ref, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
+    f = case.fresh[l]
+    out, _, _, _ = _run_lists(case, s, l, [case.sets[b].u_pos for b in range(case.w.n_req)],
+                              [case.sets[b].positions(l) for b in range(case.w.n_req)], fresh=(f.q_new, f.k_new, f.v_new))
+    assert torch.equal(out, ref)
+
+
+@pytest.mark.parametrize("variant", ["global_targets", "layerwise_sparse", "global_sparse"])
+def test_controlled_configurations_match_oracle(case, variant):
+    w = case.w
+    rng = np.random.default_rng(5)
+    s = case.make_session()
+    l = 0
+    ctx_lists, tgt_lists = [], []
+    for b in range(w.n_req):
+        T, st = w.ctx_lens[b], case.sets[b]
+        n_u = len(st.u_pos)
+        if variant == "global_targets":          # targets ranked over the whole context, not a subset of U
+            g = orc.mean_scores(np.stack([orc.minmax(case.raw[(ll, b)]) for ll in range(w.n_layers)]))
+            tgt = orc.topk(g, min(max(1, int(0.2 * T)), n_u))
+            if T > 8:
+                tgt = np.unique(np.concatenate([[0], tgt])) if st.u_pos[0] > 0 else tgt      # a target before all of U
+            ctx = st.u_pos
+        elif variant == "layerwise_sparse":      # U_l = top-|U| of this layer's score; the method's targets
+            ctx = orc.topk(case.raw[(l, b)], n_u)
+            tgt = st.positions(l)
+        else:                                    # one shared context set from the across-layer mean score
+            g = orc.mean_scores(np.stack([orc.minmax(case.raw[(ll, b)]) for ll in range(w.n_layers)]))
+            ctx = orc.topk(g, n_u)
+            tgt = st.positions(l)
+        ctx_lists.append(np.asarray(ctx, dtype=np.int32)); tgt_lists.append(np.asarray(tgt, dtype=np.int32))
+    out, lse, fresh, tcu = _run_lists(case, s, l, ctx_lists, tgt_lists)
+    for b in range(w.n_req):
+        lo, hi = int(tcu[b]), int(tcu[b + 1])
+        if hi == lo:
+            continue
+        qn, kn, vn = (inputs.bf16_bits(t[lo:hi]) for t in fresh)
+        ref, ref_lse = orc.list_attention(case.req_k(l, b), case.req_v(l, b), qn, kn, vn, ctx_lists[b], tgt_lists[b], case.scale)
+        mx, mean = attention_errors(out[lo:hi], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (variant, b, mx, mean)
+        got_lse = lse[:, lo:hi].cpu().numpy().astype(np.float64).T
+        empty = np.isneginf(ref_lse)
+        assert np.array_equal(np.isneginf(got_lse), empty)
+        np.testing.assert_allclose(got_lse[~empty], ref_lse[~empty], atol=2e-3, rtol=1e-4)
+    # cache update for the explicit target list, bit-exact
+    k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+    tgt_pos, tgt_cu, _ = _pack(tgt_lists, case.device)
+    B().relaxkv_scatter_kv_lists(s.shape, B().CacheView(k2, v2, [int(x) for x in case.ctx_cu[:-1]]), fresh[1], fresh[2],
+                                 tgt_pos, tgt_cu, [len(x) for x in tgt_lists])
+    assert_status_ok()
+    k2_b, v2_b = inputs.bf16_bits(k2), inputs.bf16_bits(v2)
+    for b in range(w.n_req):
+        lo, hi = int(tcu[b]), int(tcu[b + 1])
+        rk, rv = case.req_k(l, b).copy(), case.req_v(l, b).copy()
+        orc.scatter(rk, rv, inputs.bf16_bits(fresh[1][lo:hi]), inputs.bf16_bits(fresh[2][lo:hi]), tgt_lists[b])
+        np.testing.assert_array_equal(k2_b[case.ctx_cu[b]:case.ctx_cu[b + 1]], rk)
+        np.testing.assert_array_equal(v2_b[case.ctx_cu[b]:case.ctx_cu[b + 1]], rv)
+
+
+def test_mean_scores_and_global_topk(case):
+    """g = mean over layers of the normalised scores (fixed summation order), then top-m of g."""
+    w = case.w
+    s = case.make_session(want_norm=True)
+    s.score_select(case.q_layers, case.cache_views())
+    g = torch.empty(int(case.ctx_cu[-1]), dtype=torch.float32, device=case.device)
+    B().relaxkv_mean_scores(s.shape, w.n_layers, s.norm, g)
+    norm = s.norm.cpu().numpy()
+    ref = norm[0].astype(np.float32).copy()
+    for l in range(1, w.n_layers):
+        ref = ref + norm[l]
+    ref = ref / np.float32(w.n_layers)
+    np.testing.assert_array_equal(g.cpu().numpy(), ref)                      # same fp32 operations, same order
+    m = [max(1, t // 5) for t in w.ctx_lens]
+    anchors = torch.empty(1, sum(m), dtype=torch.int32, device=case.device)
+    B().relaxkv_select_topk(s.shape, 1, m, g.view(1, -1), anchors)
+    assert_status_ok()
+    got = anchors.cpu().numpy()[0]
+    off = 0
+    for b in range(w.n_req):
+        seg = ref[case.ctx_cu[b]:case.ctx_cu[b + 1]].astype(np.float64)
+        np.testing.assert_array_equal(got[off:off + m[b]], orc.topk(seg, m[b]))
+        off += m[b]
