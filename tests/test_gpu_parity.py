@@ -466,3 +466,47 @@ def test_mean_scores_and_global_topk(case):
         seg = ref[case.ctx_cu[b]:case.ctx_cu[b + 1]].astype(np.float64)
         np.testing.assert_array_equal(got[off:off + m[b]], orc.topk(seg, m[b]))
         off += m[b]
+
+
+# ------------------------------------------- query prefill attention feeding the scoring ----
+
+def test_query_prefill_lse_replaces_the_statistics_pass():
+    """The query's own causal attention over [context, query] (the explicit-list call with every position
+    as context and the query positions as targets, cache-only) yields each row's log-normaliser; given to
+    relaxkv_score_select it skips the statistics pass and the scores are the attention weights of that
+    wider softmax restricted to the context (the 'real forward pass' reading of the score)."""
+    w = small_qwen(n_layers=1, ctx=(1100,), q=(40,))
+    case = Case(w)
+    T, Qn, H, Hkv, D = w.ctx_lens[0], w.q_lens[0], w.n_q_heads, w.n_kv_heads, w.head_dim
+    g = torch.Generator(device="cpu").manual_seed(99)
+    kq = torch.randn(Qn, Hkv, D, generator=g).to(torch.bfloat16).to(case.device)      # the query tokens' own K/V
+    vq = torch.randn(Qn, Hkv, D, generator=g).to(torch.bfloat16).to(case.device)
+    k_ext = torch.cat([case.k_cache[0], kq]).contiguous()
+    v_ext = torch.cat([case.v_cache[0], vq]).contiguous()
+    shape_ext = B().Shape(H, Hkv, D, [T + Qn], [Qn], case.scale)
+    ws = torch.empty(B().relaxkv_workspace_bytes(shape_ext, 1) + 256, dtype=torch.uint8, device=case.device)
+    ws = ws[(-ws.data_ptr()) % 256:]
+    ctx_pos = torch.arange(T + Qn, dtype=torch.int32, device=case.device)
+    tgt_pos = torch.arange(T, T + Qn, dtype=torch.int32, device=case.device)
+    cu_ctx = torch.tensor([0, T + Qn], dtype=torch.int32, device=case.device)
+    cu_tgt = torch.tensor([0, Qn], dtype=torch.int32, device=case.device)
+    q = case.q_layers[0]
+    out = torch.empty_like(q)
+    lse = torch.empty(H, Qn, dtype=torch.float32, device=case.device)
+    B().relaxkv_list_attention(shape_ext, B().CacheView(k_ext, v_ext, [0]), q, None, None, ctx_pos, cu_ctx, tgt_pos, cu_tgt,
+                               [Qn], [T + Qn], out, ws, lse_out=lse)
+    assert_status_ok()
+    # oracle: the same causal attention, then scores with its log-normalisers
+    kb, vb, qb = inputs.bf16_bits(k_ext), inputs.bf16_bits(v_ext), inputs.bf16_bits(q)
+    ref_out, ref_lse = orc.list_attention(kb, vb, qb, None, None, np.arange(T + Qn), np.arange(T, T + Qn), case.scale)
+    mx, mean = attention_errors(out, ref_out)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS
+    np.testing.assert_allclose(lse.cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+    ref_raw = orc.raw_scores(qb, kb[:T], case.scale, lse=ref_lse.T)
+    s = case.make_session()
+    s.score_select(case.q_layers, case.cache_views(), row_lse_layers=[lse])
+    assert_status_ok()
+    got = s.raw.cpu().numpy()[0].astype(np.float64)
+    assert np.all(np.abs(got - ref_raw) <= 1e-3 * ref_raw + 1e-6 / T)
+    assert got.sum() < 1.0                                   # part of each row's mass sits on the query's own keys
+    check_anchor_band(ref_raw, case.k[0], s.anchors.cpu().numpy()[0])
