@@ -117,7 +117,9 @@ size_t relaxkv_workspace_bytes(const relaxkv_shape* shape, int32_t n_layers, con
  * h_k              host [B]: anchors per layer for each request, 1 <= k_b <= T_c.
  * raw_scores_out   device fp32 [n_layers, sum_b T_c].
  * norm_scores_out  NULL or device fp32 [n_layers, sum_b T_c].
- * anchors_out      device int32 [n_layers, sum_b k_b]; request-local positions.
+ * anchors_out      device int32 [n_layers, sum_b k_b]; request-local positions.  NULL: scoring only (no
+ *                  selection, norm_scores_out is not written) - for callers that first combine the scores
+ *                  of several head shards (mean over shards of equal size) and then call relaxkv_select_topk.
  * Results are deterministic: reductions run in a fixed order (no floating-point atomics).
  */
 relaxkv_status relaxkv_score_select(

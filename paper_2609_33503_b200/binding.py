@@ -146,7 +146,7 @@ def relaxkv_workspace_bytes(shape: Shape, n_layers: int, k: Optional[Sequence[in
 
 
 def relaxkv_score_select(shape: Shape, q_layers: List[torch.Tensor], cache_layers: List[CacheView],
-                         k: Sequence[int], raw_scores_out: torch.Tensor, anchors_out: torch.Tensor,
+                         k: Sequence[int], raw_scores_out: torch.Tensor, anchors_out: Optional[torch.Tensor],
                          workspace: torch.Tensor, norm_scores_out: Optional[torch.Tensor] = None,
                          row_lse_layers: Optional[List[Optional[torch.Tensor]]] = None, stream=None) -> None:
     n_layers = len(q_layers)

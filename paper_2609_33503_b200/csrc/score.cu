@@ -80,8 +80,7 @@ extern "C" relaxkv_status relaxkv_score_select(
     void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
-  if (n_layers < 1 || !q_layers || !cache_layers || !h_k || !raw_scores_out || !anchors_out || !workspace ||
-      !shape->h_q_len)
+  if (n_layers < 1 || !q_layers || !cache_layers || !h_k || !raw_scores_out || !workspace || !shape->h_q_len)
     return RELAXKV_ERR_INVALID_ARG;
   for (int b = 0; b < shape->n_req; ++b) {
     if (shape->h_q_len[b] < 1) return RELAXKV_ERR_INVALID_ARG;
@@ -109,6 +108,7 @@ extern "C" relaxkv_status relaxkv_score_select(
       rc = score_layer<64>(shape, rt, plan, q_layers[l], &cache_layers[l], lse, raw, static_cast<char*>(workspace), ws, stream);
     if (rc != RELAXKV_OK) return rc;
   }
+  if (!anchors_out) return RELAXKV_OK;      // scoring only: the caller reduces the scores first (head-sharded serving)
   ReqTable rt;
   fill_req_table(rt, shape, nullptr, h_k);
   return launch_select(rt, n_layers, raw_scores_out, norm_scores_out, anchors_out, stream);

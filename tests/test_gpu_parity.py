@@ -510,3 +510,34 @@ def test_query_prefill_lse_replaces_the_statistics_pass():
     assert np.all(np.abs(got - ref_raw) <= 1e-3 * ref_raw + 1e-6 / T)
     assert got.sum() < 1.0                                   # part of each row's mass sits on the query's own keys
     check_anchor_band(ref_raw, case.k[0], s.anchors.cpu().numpy()[0])
+
+
+def test_head_sharded_selection_on_one_gpu():
+    """The head-sharded selection path, its ranks run one after the other on this GPU (their kernels never wait
+    on one another): partial scores of the two KV-head shards average to the unsharded scores, and the anchors
+    computed from the combined scores are those of the unsharded call."""
+    from paper_2609_33503_b200 import sharded
+    from paper_2609_33503_b200.pipeline import RepairSession
+    case = Case(small_llama(n_layers=2, ctx=(1536,), q=(24,)))
+    w = case.w
+    full = case.make_session()
+    full.score_select(case.q_layers, case.cache_views())
+    world = 2
+    parts = []
+    for rank in range(world):
+        kv_lo, kv_hi, q_lo, q_hi = sharded.head_shard(w.n_q_heads, w.n_kv_heads, world, rank)
+        s = RepairSession(q_hi - q_lo, kv_hi - kv_lo, w.head_dim, w.ctx_lens, w.q_lens, w.n_layers, case.k,
+                          device=case.device, softmax_scale=case.scale)
+        qs = [q[:, q_lo:q_hi].contiguous() for q in case.q_layers]
+        views = [B().CacheView(k[:, kv_lo:kv_hi], v[:, kv_lo:kv_hi], [0]) for k, v in zip(case.k_cache, case.v_cache)]
+        sharded.sharded_score_select(s, qs, views, world=1)          # world=1: no process group on this box
+        parts.append(s.raw.clone())
+    combined = (parts[0] + parts[1]) / world
+    assert_status_ok()
+    torch.testing.assert_close(combined, full.raw, rtol=2e-5, atol=1e-9)
+    s0 = RepairSession(w.n_q_heads // world, w.n_kv_heads // world, w.head_dim, w.ctx_lens, w.q_lens, w.n_layers, case.k,
+                       device=case.device, softmax_scale=case.scale)
+    anchors = torch.empty_like(full.anchors)
+    B().relaxkv_select_topk(s0.shape, w.n_layers, case.k, combined, anchors)
+    for l in range(w.n_layers):
+        check_anchor_band(case.raw[(l, 0)], case.k[0], anchors[l].cpu().numpy())
