@@ -109,6 +109,26 @@ constexpr int kScoreMaxRows = 640;    // query rows (token x head-in-group) resi
 constexpr int kScoreTokBox = 8;       // query tokens per TMA box of the scoring kernel
 constexpr int kCtxPadRows = 128;      // zero rows after the materialised context
 
+constexpr int kScoreLayersPerLaunch = 48;   // layers scored by one launch (their tensor maps travel as parameters)
+
+// Key-range splits for a launch that scores `layers` layers at once: at least two waves of CTAs on the 148
+// SMs (one CTA per SM), and a count that fills its last wave (every CTA of a launch does the same work).
+inline int score_splits(long long units_times_heads, int layers) {
+  const long long per = units_times_heads * layers;
+  if (per <= 0) return 1;
+  int best = 1;
+  double best_eff = 0.0;
+  for (int ns = 1; ns <= kScoreSplitsMax; ++ns) {
+    const long long ctas = per * ns;
+    if (ctas < 2 * 148 && ns < kScoreSplitsMax) continue;
+    const long long waves = (ctas + 147) / 148;
+    const double eff = (double)ctas / (double)(waves * 148);
+    if (eff > best_eff + 0.02) { best_eff = eff; best = ns; }      // prefer fewer, longer CTAs unless clearly better
+    if (ctas >= 16 * 148) break;
+  }
+  return best;
+}
+
 // Query-row blocks a request needs so that each block's rows fit resident (scoring kernel).
 inline int score_blocks(int q_len, int group) {
   const int max_tok = kScoreMaxRows / group / kScoreTokBox * kScoreTokBox;
@@ -120,7 +140,8 @@ struct WsLayout {
   size_t kctx, vctx; long long ctx_rows_cap;
   // explicit-list attention: limit [sumT] i32 | fresh_row [sumT] i32
   size_t list_limit, list_fresh;
-  // scoring: lse [H, sumQ] f32 | part [2*kScoreSplitsMax, H, sumQ] float2 | colpart [2*H_kv*max_blocks, sumT] f32
+  // scoring (per launch of Lc <= kScoreLayersPerLaunch layers): lse [Lc, H, sumQ] f32 |
+  // part [Lc, 2*n_splits, H, sumQ] float2 | colpart [Lc, 2*H_kv*max_blocks, sumT] f32
   size_t lse, part, colpart;
   // sets: counts [B + L*B] i32
   size_t counts;
@@ -140,14 +161,22 @@ inline WsLayout ws_layout(const relaxkv_shape* s, int n_layers) {
   w.list_fresh = a; a = align_up(a + (size_t)sum_t * 4, 256);
   size_t attn_total = a;
   a = 0;
-  w.lse = a; a = align_up(a + (size_t)s->n_q_heads * sum_q * 4, 256);
+  const int lc_max = n_layers < kScoreLayersPerLaunch ? n_layers : kScoreLayersPerLaunch;
+  w.lse = a; a = align_up(a + (size_t)lc_max * s->n_q_heads * sum_q * 4, 256);
   int max_blocks = 1;
   for (int b = 0; b < s->n_req; ++b) {
     const int nb = score_blocks(s->h_q_len ? s->h_q_len[b] : 0, s->n_q_heads / s->n_kv_heads);
     if (nb > max_blocks) max_blocks = nb;
   }
-  w.part = a; a = align_up(a + (size_t)2 * kScoreSplitsMax * s->n_q_heads * sum_q * 8, 256);
-  w.colpart = a; a = align_up(a + (size_t)2 * s->n_kv_heads * max_blocks * sum_t * 4, 256);
+  long long units = 0;
+  for (int b = 0; b < s->n_req; ++b) units += score_blocks(s->h_q_len ? s->h_q_len[b] : 0, s->n_q_heads / s->n_kv_heads);
+  long long part_slots = 1;                 // max over launch sizes of layers x 2 x splits
+  for (int lc = 1; lc <= lc_max; ++lc) {
+    const long long v = (long long)lc * 2 * score_splits(units * s->n_kv_heads, lc);
+    if (v > part_slots) part_slots = v;
+  }
+  w.part = a; a = align_up(a + (size_t)part_slots * s->n_q_heads * sum_q * 8, 256);
+  w.colpart = a; a = align_up(a + (size_t)lc_max * 2 * s->n_kv_heads * max_blocks * sum_t * 4, 256);
   size_t score_total = a;
   w.counts = 0;
   size_t sets_total = align_up((size_t)(s->n_req + (size_t)n_layers * s->n_req + 2) * 4, 256);

@@ -13,58 +13,71 @@ namespace relaxkv {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-// lse[h, row] = ln sum over the partial (max, sum) pairs (log2 units in, natural log out).
-__global__ void combine_lse_kernel(int H, int sum_q, int n_part, const float2* __restrict__ part,
+// lse[layer, h, row] = ln sum over the partial (max, sum) pairs (log2 units in, natural log out).
+// One warp per row: the lanes walk the partials (fixed lane -> partial assignment, fixed shuffle tree, so
+// the result does not depend on scheduling).  part is [layer][n_part][H*sum_q].  Rows of layers whose
+// log-normalisers were supplied have only empty partials and are never read afterwards.
+__global__ void combine_lse_kernel(long long n_rows_total, long long n_rows, int n_part, const float2* __restrict__ part,
                                    float* __restrict__ lse) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= H * sum_q) return;
+  const int lane = threadIdx.x & 31;
+  const long long gidx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (gidx >= n_rows_total) return;
+  const long long layer = gidx / n_rows, idx = gidx - layer * n_rows;
+  const float2* pl = part + layer * n_part * n_rows;
   float M = -INFINITY;
-  for (int s = 0; s < n_part; ++s) {
-    const float2 p = part[(long long)s * H * sum_q + idx];
+  for (int s = lane; s < n_part; s += 32) {
+    const float2 p = pl[(long long)s * n_rows + idx];
     if (p.y > 0.f) M = fmaxf(M, p.x);
   }
+  M = warp_reduce_max(M);
   float z = 0.f;
-  for (int s = 0; s < n_part; ++s) {
-    const float2 p = part[(long long)s * H * sum_q + idx];
+  for (int s = lane; s < n_part; s += 32) {
+    const float2 p = pl[(long long)s * n_rows + idx];
     if (p.y > 0.f) z += p.y * exp2f(p.x - M);
   }
-  lse[idx] = (M + log2f(z)) * kLn2;
+  z = warp_reduce_sum(z);
+  if (lane == 0) lse[gidx] = (M + log2f(z)) * kLn2;
 }
 
-void launch_combine_lse(int H, int sum_q, int n_part, const float2* part, float* lse, cudaStream_t stream) {
-  combine_lse_kernel<<<(H * sum_q + 255) / 256, 256, 0, stream>>>(H, sum_q, n_part, part, lse);
+void launch_combine_lse(int n_layers, int H, int sum_q, int n_part, const float2* part, float* lse, cudaStream_t stream) {
+  const long long n_rows = (long long)H * sum_q, total = n_rows * n_layers;
+  combine_lse_kernel<<<(unsigned)((total * 32 + 255) / 256), 256, 0, stream>>>(total, n_rows, n_part, part, lse);
 }
 
-// raw[i] = (sum of the partial column sums in a fixed order: KV head, query-row block, warpgroup) / (H * Q_b)
-// rt.tile_cu = prefix of the query-row blocks per request.
-__global__ void finalize_raw_kernel(ReqTable rt, int H, int Hkv, int max_super, const float* __restrict__ colpart,
-                                    float* __restrict__ raw) {
+// raw[layer, i] = (sum of the partial column sums in a fixed order: KV head, query-row block, warpgroup) / (H * Q_b)
+// rt.tile_cu = prefix of the query-row blocks per request; colpart is [layer][2*Hkv*max_super][sum_t].
+__global__ void finalize_raw_kernel(ReqTable rt, int n_layers, int H, int Hkv, int max_super,
+                                    const float* __restrict__ colpart, float* __restrict__ raw) {
   const long long sum_t = rt.ctx_cu[rt.n_req];
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= sum_t) return;
+  const long long gi = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gi >= sum_t * n_layers) return;
+  const long long layer = gi / sum_t, i = gi - layer * sum_t;
   int b = 0;
   while (b + 1 < rt.n_req && i >= rt.ctx_cu[b + 1]) ++b;
   const int n_super = rt.tile_cu[b + 1] - rt.tile_cu[b];
+  const float* cp = colpart + layer * (2 * Hkv * max_super) * sum_t;
   float s = 0.f;
   for (int g = 0; g < Hkv; ++g)
     for (int sp = 0; sp < n_super; ++sp)
-      for (int w = 0; w < 2; ++w) s += colpart[(long long)((g * max_super + sp) * 2 + w) * sum_t + i];
-  raw[i] = s / ((float)H * (float)rt.q_len[b]);
+      for (int w = 0; w < 2; ++w) s += cp[(long long)((g * max_super + sp) * 2 + w) * sum_t + i];
+  raw[gi] = s / ((float)H * (float)rt.q_len[b]);
 }
 
 template <int D>
-static relaxkv_status score_layer(const relaxkv_shape* shape, ReqTable rt, const ScorePlan& plan, const void* q,
-                                  const relaxkv_cache_view* cache, const float* lse_given, float* raw,
-                                  char* workspace, const WsLayout& ws, cudaStream_t stream) {
+static relaxkv_status score_layers(const relaxkv_shape* shape, ReqTable rt, const ScorePlan& plan, int n_layers,
+                                   const void* const* q_layers, const relaxkv_cache_view* cache_layers,
+                                   const float* const* lse_given, float* raw, char* workspace, const WsLayout& ws,
+                                   cudaStream_t stream) {
   const int B = shape->n_req, H = shape->n_q_heads, Hkv = shape->n_kv_heads;
   float* lse_ws = reinterpret_cast<float*>(workspace + ws.lse);
   float2* part = reinterpret_cast<float2*>(workspace + ws.part);
   float* colpart = reinterpret_cast<float*>(workspace + ws.colpart);
-  relaxkv_status rc = launch_score_sm100<D>(shape, rt, plan, q, cache, lse_given, lse_ws, part, colpart, stream);
+  relaxkv_status rc = launch_score_sm100<D>(shape, rt, plan, n_layers, q_layers, cache_layers, lse_given, lse_ws, part,
+                                            colpart, stream);
   if (rc != RELAXKV_OK) return rc;
   for (int b = 0; b < B; ++b) rt.tile_cu[b + 1] = rt.tile_cu[b] + plan.n_super[b];
-  const long long sum_t = rt.ctx_cu[B];
-  finalize_raw_kernel<<<(unsigned)((sum_t + 255) / 256), 256, 0, stream>>>(rt, H, Hkv, plan.max_super, colpart, raw);
+  const long long total = rt.ctx_cu[B] * n_layers;
+  finalize_raw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(rt, n_layers, H, Hkv, plan.max_super, colpart, raw);
   return launch_ok();
 }
 
@@ -97,16 +110,27 @@ extern "C" relaxkv_status relaxkv_score_select(
   for (int b = 0; b < shape->n_req; ++b) sum_t += shape->h_ctx_len[b];
 
   const ScorePlan plan = plan_score(shape);
-  for (int l = 0; l < n_layers; ++l) {
+  // Layers are scored in groups: one launch per pass covers up to kScoreLayersPerLaunch consecutive layers whose
+  // cache views place the requests at the same token offsets (the usual case: all of them).
+  for (int l0 = 0; l0 < n_layers;) {
+    int l1 = l0 + 1;
+    while (l1 < n_layers && l1 - l0 < kScoreLayersPerLaunch) {
+      bool same = true;
+      for (int b = 0; b < shape->n_req; ++b)
+        same = same && cache_layers[l1].h_req_token_offset[b] == cache_layers[l0].h_req_token_offset[b];
+      if (!same) break;
+      ++l1;
+    }
     ReqTable rt;
-    fill_req_table(rt, shape, &cache_layers[l], h_k);
-    const float* lse = row_lse_layers ? row_lse_layers[l] : nullptr;
-    float* raw = raw_scores_out + (long long)l * sum_t;
+    fill_req_table(rt, shape, &cache_layers[l0], h_k);
+    const float* const* lse = row_lse_layers ? row_lse_layers + l0 : nullptr;
+    float* raw = raw_scores_out + (long long)l0 * sum_t;
     if (shape->head_dim == 128)
-      rc = score_layer<128>(shape, rt, plan, q_layers[l], &cache_layers[l], lse, raw, static_cast<char*>(workspace), ws, stream);
+      rc = score_layers<128>(shape, rt, plan, l1 - l0, q_layers + l0, cache_layers + l0, lse, raw, static_cast<char*>(workspace), ws, stream);
     else
-      rc = score_layer<64>(shape, rt, plan, q_layers[l], &cache_layers[l], lse, raw, static_cast<char*>(workspace), ws, stream);
+      rc = score_layers<64>(shape, rt, plan, l1 - l0, q_layers + l0, cache_layers + l0, lse, raw, static_cast<char*>(workspace), ws, stream);
     if (rc != RELAXKV_OK) return rc;
+    l0 = l1;
   }
   if (!anchors_out) return RELAXKV_OK;      // scoring only: the caller reduces the scores first (head-sharded serving)
   ReqTable rt;

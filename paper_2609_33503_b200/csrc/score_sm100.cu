@@ -7,7 +7,7 @@
 //   pass 1 (row statistics):  S   = Q_chunk K_tile^T   lanes = query rows, columns = keys
 //   pass 2 (column sums):     S^T = K_tile Q_chunk^T   lanes = keys,       columns = query rows
 // so that in both passes the reduction a thread needs runs along its own TMEM lane.  Two softmax
-// warpgroups split the 128 columns of every buffer; the exponentials (one per 2*D MMA flops) bound the
+// warpgroups take the buffers alternately; the exponentials (one per 2*D MMA flops) bound the
 // kernel, not the tensor pipe and not HBM.  Partial results are combined in a fixed order by the
 // small kernels of score.cu, so scores are bit-reproducible.
 #include "score_sm100.cuh"
@@ -36,12 +36,19 @@ struct ScoreSmem {
   static constexpr int kTotal = kMisc + 16;
 };
 
+// Per-layer arguments of one launch: tensor maps of the layer's Q rows and K cache, its supplied
+// log-normalisers (NULL: computed by pass 1) - by value in the kernel parameters.
+struct ScoreLayers {
+  CUtensorMap tm_q[kScoreLayersPerLaunch];
+  CUtensorMap tm_k[kScoreLayersPerLaunch];
+  const float* lse_given[kScoreLayersPerLaunch];
+};
+
 template <int D, bool PASS2>
 __global__ void __launch_bounds__(kScThreads, 1)
-score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ ReqTable rt, int H, int Hkv, float scale_log2, int n_splits,
-                   int max_super, const float* __restrict__ lse, float2* __restrict__ part,
-                   float* __restrict__ colpart, DeviceStatus* st) {
+score_sm100_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ ReqTable rt, int H, int Hkv,
+                   float scale_log2, int n_splits, int max_super, const float* __restrict__ lse_ws,
+                   float2* __restrict__ part_all, float* __restrict__ colpart_all, DeviceStatus* st) {
   using L = ScoreSmem<D>;
   constexpr int kHalves = L::kHalves;
   constexpr float kLog2e = 1.4426950408889634f;
@@ -49,7 +56,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   // ---- which unit ---------------------------------------------------------------------------------
   const int B = rt.n_req;
   const int G = H / Hkv;
-  const int g = blockIdx.y, split = blockIdx.z;
+  const int layer = blockIdx.z / n_splits, split = blockIdx.z - layer * n_splits;
+  const int g = blockIdx.y;
   const int b = find_segment(rt.tile_cu, B, (int)blockIdx.x);     // rt.tile_cu: prefix of query-row blocks
   const int super = blockIdx.x - rt.tile_cu[b];
   const int n_super = rt.tile_cu[b + 1] - rt.tile_cu[b];
@@ -67,6 +75,13 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int kt0 = split * per, kt1 = min(n_kt, kt0 + per);
   const int sum_q = rt.q_cu[B];
   const long long sum_t = rt.ctx_cu[B];
+  const CUtensorMap& tm_q = layers.tm_q[layer];
+  const CUtensorMap& tm_k = layers.tm_k[layer];
+  const float* given = layers.lse_given[layer];
+  if (!PASS2 && given != nullptr) return;                          // this layer's log-normalisers were supplied
+  const float* lse = given ? given : lse_ws + (long long)layer * H * sum_q;
+  float2* part = part_all + (long long)layer * (2 * n_splits) * H * sum_q;
+  float* colpart = colpart_all + (long long)layer * (2 * Hkv * max_super) * sum_t;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = warp >> 2;                                        // softmax warpgroup (0/1) for warps 0..7
   const int lane_row = (warp & 3) * 32 + lane;                     // TMEM lane of a softmax thread
@@ -105,7 +120,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
     for (int s = 0; s < kScKStages; ++s) { mbar_init(bar_kfull + 8 * s, 1); mbar_init(bar_kempty + 8 * s, 1); }
-    for (int i = 0; i < kScBufs; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, 256); }
+    for (int i = 0; i < kScBufs; ++i) { mbar_init(bar_sfull + 8 * i, 1); mbar_init(bar_sempty + 8 * i, 128); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -178,8 +193,10 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     }
   } else {
-    // ================= softmax warpgroups: each takes 64 of the 128 columns of every buffer =================
-    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + wg * 64;
+    // ================= softmax warpgroups: warpgroup w consumes the buffers of items it % 2 == w =================
+    // (whole 128-column buffers: one barrier wait - ~145 cycles even when it succeeds at once - per 128
+    //  exponentials of a thread instead of per 64)
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     float m_row[kScoreMaxRows / 128], z_row[kScoreMaxRows / 128];
 #pragma unroll
     for (int c = 0; c < kScoreMaxRows / 128; ++c) { m_row[c] = -INFINITY; z_row[c] = 0.f; }
@@ -190,50 +207,58 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
       for (int c = 0; c < kScoreMaxRows / 128; ++c) {
         if (c < n_chunks) {
-          const int buf = it % kScBufs;
-          ok = mbar_wait(bar_sfull + 8 * buf, (it / kScBufs) & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
-          uint32_t s[64];
-          tmem_ld32(t_lane + buf * 128, &s[0]);
-          tmem_ld32(t_lane + buf * 128 + 32, &s[32]);
-          tmem_wait_ld();
-          tc_fence_before();
-          mbar_arrive(bar_sempty + 8 * buf);                        // the values are in registers: release the buffer
-          ++it;
-          if (PASS2) {
-            const float4* l4 = reinterpret_cast<const float4*>(lse2s + c * 128 + wg * 64);
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          const int my_it = it++;
+          if ((my_it & 1) == wg) {
+            const int buf = my_it % kScBufs;
+            ok = mbar_wait(bar_sfull + 8 * buf, (my_it / kScBufs) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t s[128];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float4 lv = l4[i];
-              a0 += fast_exp2(fmaf(__uint_as_float(s[4 * i]), scale_log2, -lv.x));
-              a1 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 1]), scale_log2, -lv.y));
-              a2 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 2]), scale_log2, -lv.z));
-              a3 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 3]), scale_log2, -lv.w));
-            }
-            acc += (a0 + a1) + (a2 + a3);
-          } else {
-            const int key0 = kt * 128 + wg * 64;
-            if (key0 + 63 >= T) {
+            for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(t_lane + buf * 128 + q4 * 32, &s[q4 * 32]);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar_sempty + 8 * buf);                      // the values are in registers: release the buffer
+            if (PASS2) {
+              const float4* l4 = reinterpret_cast<const float4*>(lse2s + c * 128);
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-              for (int i = 0; i < 64; ++i)
-                if (key0 + i >= T) s[i] = 0xff800000u;               // keys past the context: -inf
-            }
-            float mx = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
-            const float m_new = fmaxf(m_row[c], mx * scale_log2);
-            if (m_new > -INFINITY) {
-              float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-              for (int i = 0; i < 64; i += 2) {
-                a0 += fast_exp2(fmaf(__uint_as_float(s[i]), scale_log2, -m_new));
-                a1 += fast_exp2(fmaf(__uint_as_float(s[i + 1]), scale_log2, -m_new));
+              for (int i = 0; i < 32; ++i) {
+                const float4 lv = l4[i];
+                a0 += fast_exp2(fmaf(__uint_as_float(s[4 * i]), scale_log2, -lv.x));
+                a1 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 1]), scale_log2, -lv.y));
+                a2 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 2]), scale_log2, -lv.z));
+                a3 += fast_exp2(fmaf(__uint_as_float(s[4 * i + 3]), scale_log2, -lv.w));
               }
-              z_row[c] = z_row[c] * fast_exp2(m_row[c] - m_new) + (a0 + a1);
-              m_row[c] = m_new;
+              acc += (a0 + a1) + (a2 + a3);
+            } else {
+              const int key0 = kt * 128;
+              if (key0 + 127 >= T) {
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                  if (key0 + i >= T) s[i] = 0xff800000u;             // keys past the context: -inf
+              }
+              float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+              for (int i = 0; i < 128; i += 4) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], __uint_as_float(s[i + e]));
+              }
+              const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+              const float m_new = fmaxf(m_row[c], mx * scale_log2);
+              if (m_new > -INFINITY) {
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 128; i += 4) {
+                  a0 += fast_exp2(fmaf(__uint_as_float(s[i]), scale_log2, -m_new));
+                  a1 += fast_exp2(fmaf(__uint_as_float(s[i + 1]), scale_log2, -m_new));
+                  a2 += fast_exp2(fmaf(__uint_as_float(s[i + 2]), scale_log2, -m_new));
+                  a3 += fast_exp2(fmaf(__uint_as_float(s[i + 3]), scale_log2, -m_new));
+                }
+                z_row[c] = z_row[c] * fast_exp2(m_row[c] - m_new) + ((a0 + a1) + (a2 + a3));
+                m_row[c] = m_new;
+              }
             }
           }
         }
@@ -288,21 +313,17 @@ ScorePlan plan_score(const relaxkv_shape* shape) {
     p.units += ns;
     if (ns > p.max_super) p.max_super = ns;
   }
-  const long long ctas_wanted = 2 * 148;
-  long long per_split = (long long)p.units * shape->n_kv_heads;
-  int ns = per_split > 0 ? (int)((ctas_wanted + per_split - 1) / per_split) : 1;
-  if (ns < 1) ns = 1;
-  if (ns > kScoreSplitsMax) ns = kScoreSplitsMax;
-  p.n_splits = ns;
   return p;
 }
 
 template <int D>
-relaxkv_status launch_score_sm100(const relaxkv_shape* shape, ReqTable rt, const ScorePlan& plan, const void* q,
-                                  const relaxkv_cache_view* cache, const float* lse_given, float* lse_ws,
-                                  float2* part, float* colpart, cudaStream_t stream) {
+relaxkv_status launch_score_sm100(const relaxkv_shape* shape, ReqTable rt, const ScorePlan& plan, int n_layers,
+                                  const void* const* q_layers, const relaxkv_cache_view* cache_layers,
+                                  const float* const* lse_given, float* lse_ws, float2* part, float* colpart,
+                                  cudaStream_t stream) {
   const int B = shape->n_req, H = shape->n_q_heads, Hkv = shape->n_kv_heads, G = H / Hkv;
   const int sum_q = rt.q_cu[B];
+  if (n_layers < 1 || n_layers > kScoreLayersPerLaunch) return RELAXKV_ERR_INVALID_ARG;
   long long tok_extent = 0;
   for (int b = 0; b < B; ++b) {
     rt.tile_cu[b + 1] = rt.tile_cu[b] + plan.n_super[b];
@@ -310,34 +331,52 @@ relaxkv_status launch_score_sm100(const relaxkv_shape* shape, ReqTable rt, const
     if (e > tok_extent) tok_extent = e;
   }
   if (tok_extent > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap tm_q, tm_k;
-  if (!make_map_3d(&tm_q, q, D, H, (uint64_t)sum_q, (uint64_t)D * 2, (uint64_t)H * D * 2, (uint32_t)G, kScTokBox) ||
-      !make_map_3d(&tm_k, cache->k, D, Hkv, (uint64_t)tok_extent, (uint64_t)cache->head_stride * 2,
-                   (uint64_t)cache->token_stride * 2, 1u, 128u))
-    return RELAXKV_ERR_CUDA;
+  ScoreLayers layers;
+  bool need_pass1 = false;
+  for (int l = 0; l < n_layers; ++l) {
+    const relaxkv_cache_view* c = &cache_layers[l];
+    if (!make_map_3d(&layers.tm_q[l], q_layers[l], D, H, (uint64_t)sum_q, (uint64_t)D * 2, (uint64_t)H * D * 2, (uint32_t)G,
+                     kScTokBox) ||
+        !make_map_3d(&layers.tm_k[l], c->k, D, Hkv, (uint64_t)tok_extent, (uint64_t)c->head_stride * 2,
+                     (uint64_t)c->token_stride * 2, 1u, 128u))
+      return RELAXKV_ERR_CUDA;
+    layers.lse_given[l] = lse_given ? lse_given[l] : nullptr;
+    if (!layers.lse_given[l]) need_pass1 = true;
+  }
+  for (int l = n_layers; l < kScoreLayersPerLaunch; ++l) {
+    layers.tm_q[l] = layers.tm_q[0]; layers.tm_k[l] = layers.tm_k[0]; layers.lse_given[l] = nullptr;
+  }
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
   const float scale_log2 = shape->softmax_scale * 1.4426950408889634f;
-  const dim3 grid((unsigned)rt.tile_cu[B], (unsigned)Hkv, (unsigned)plan.n_splits);
+  const int n_splits = score_splits((long long)plan.units * Hkv, n_layers);
+  const dim3 grid((unsigned)rt.tile_cu[B], (unsigned)Hkv, (unsigned)(n_splits * n_layers));
   if (grid.x == 0) return RELAXKV_OK;
   constexpr int smem = ScoreSmem<D>::kTotal;
-  if (!lse_given) {
-    auto k1 = score_sm100_kernel<D, false>;
-    if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RELAXKV_ERR_CUDA;
-    k1<<<grid, kScThreads, smem, stream>>>(tm_q, tm_k, rt, H, Hkv, scale_log2, plan.n_splits, plan.max_super, nullptr,
-                                           part, nullptr, st);
-    launch_combine_lse(H, sum_q, plan.n_splits * 2, part, lse_ws, stream);
-  }
+  static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
+  auto k1 = score_sm100_kernel<D, false>;
   auto k2 = score_sm100_kernel<D, true>;
-  if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RELAXKV_ERR_CUDA;
-  k2<<<grid, kScThreads, smem, stream>>>(tm_q, tm_k, rt, H, Hkv, scale_log2, plan.n_splits, plan.max_super,
-                                         lse_given ? lse_given : lse_ws, nullptr, colpart, st);
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return RELAXKV_ERR_CUDA;
+    attr_done[dev] = true;
+  }
+  if (need_pass1) {
+    k1<<<grid, kScThreads, smem, stream>>>(layers, rt, H, Hkv, scale_log2, n_splits, plan.max_super, lse_ws, part, colpart, st);
+    launch_combine_lse(n_layers, H, sum_q, n_splits * 2, part, lse_ws, stream);
+  }
+  k2<<<grid, kScThreads, smem, stream>>>(layers, rt, H, Hkv, scale_log2, n_splits, plan.max_super, lse_ws, part, colpart, st);
   return launch_ok();
 }
 
-template relaxkv_status launch_score_sm100<64>(const relaxkv_shape*, ReqTable, const ScorePlan&, const void*,
-                                               const relaxkv_cache_view*, const float*, float*, float2*, float*, cudaStream_t);
-template relaxkv_status launch_score_sm100<128>(const relaxkv_shape*, ReqTable, const ScorePlan&, const void*,
-                                                const relaxkv_cache_view*, const float*, float*, float2*, float*, cudaStream_t);
+template relaxkv_status launch_score_sm100<64>(const relaxkv_shape*, ReqTable, const ScorePlan&, int, const void* const*,
+                                               const relaxkv_cache_view*, const float* const*, float*, float2*, float*,
+                                               cudaStream_t);
+template relaxkv_status launch_score_sm100<128>(const relaxkv_shape*, ReqTable, const ScorePlan&, int, const void* const*,
+                                                const relaxkv_cache_view*, const float* const*, float*, float2*, float*,
+                                                cudaStream_t);
 
 }  // namespace relaxkv
