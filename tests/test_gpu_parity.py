@@ -541,3 +541,32 @@ def test_head_sharded_selection_on_one_gpu():
     B().relaxkv_select_topk(s0.shape, w.n_layers, case.k, combined, anchors)
     for l in range(w.n_layers):
         check_anchor_band(case.raw[(l, 0)], case.k[0], anchors[l].cpu().numpy())
+
+
+# ------------------------------------------------ other head geometries and cache layouts ----
+
+@pytest.mark.parametrize("H,Hkv,D,head_major", [(8, 8, 128, False), (16, 8, 64, True), (16, 2, 128, False),
+                                                (32, 2, 64, False), (12, 4, 128, True)])
+def test_other_geometries_and_head_major_cache(H, Hkv, D, head_major):
+    """Group sizes 1, 2, 8, 16 and 3 (the last does not divide 128), both head dims, and a cache stored
+    [H_kv, tokens, D] (read through its strides by the TMA-based scoring kernel and by the gather)."""
+    base = inputs.Workload("geom", 2, H, Hkv, D, 64, (700, 333), (21, 9), 0.2, base_seed=7,
+                           planted_chunks=((1, 6), (2,)), variant="calibrated")
+    case = Case(base, head_major_cache=head_major)
+    w = case.w
+    s = case.make_session(want_norm=True)
+    s.score_select(case.q_layers, case.cache_views())
+    assert_status_ok()
+    raw = s.raw.cpu().numpy().astype(np.float64)
+    anchors = s.anchors.cpu().numpy()
+    for l in range(w.n_layers):
+        for b in range(w.n_req):
+            ref = case.raw[(l, b)]
+            got = raw[l, case.ctx_cu[b]:case.ctx_cu[b + 1]]
+            assert np.all(np.abs(got - ref) <= 1e-3 * ref + 1e-6 / w.ctx_lens[b]), np.abs(got / ref - 1).max()
+            check_anchor_band(ref, case.k[b], anchors[l, case.k_cu[b]:case.k_cu[b + 1]])
+    s.build_active_sets(case.anchors_tensor())
+    for l in range(w.n_layers):
+        for full_prefix in (False, True):
+            out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
+            check_attention(case, l, out, lse, full_prefix)
