@@ -280,6 +280,45 @@ relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers,
                                    float* mean_out, relaxkv_stream stream);
 
 /*
+ * ---- Dense block work of the active targets (Algorithm 1, steps 14, 16 and 20; Section 3.3 for the
+ * position IDs).  The method runs "the unchanged Transformer block" on the |R_l| active rows only; these
+ * calls are that block for a Llama-style pre-norm decoder.  All tensors bf16, row-major, 16-byte aligned,
+ * feature counts multiples of 8; fp32 arithmetic inside.  The caller owns every buffer. ----
+ */
+
+/* y[r, :] = x[r, :] * rsqrt(mean(x[r, :]^2) + eps) * weight[:]      x, y [n_rows, n_cols], weight [n_cols] */
+relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64_t n_rows, int32_t n_cols,
+                               float eps, relaxkv_stream stream);
+
+/* y = x weight^T (+ residual)      x [n_rows, n_in], weight [n_out, n_in] (the [out, in] layout),
+ * residual NULL or [n_rows, n_out], y [n_rows, n_out] (may alias residual).  tcgen05 GEMM. */
+relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
+                              int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream);
+
+/* Rotary embedding in place, rotate-half convention: pair i < D/2 of each head vector is rotated by
+ * positions[row] * theta^(-2i/D).  x [n_rows, n_heads, head_dim]; positions: device int32 [n_rows], the rows'
+ * ORIGINAL global positions (Section 3.3: restricting the context does not renumber tokens). */
+relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
+                            float theta, relaxkv_stream stream);
+
+/* out[r, i] = silu(gate_up[r, i]) * gate_up[r, n_inter + i]      gate_up [n_rows, 2*n_inter], out [n_rows, n_inter] */
+relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t n_rows, int32_t n_inter, relaxkv_stream stream);
+
+/* positions_out[row] = position of target row of this layer (row order = the layer's R lists, requests
+ * packed): u_pos[u_cu[b] + r_rank[r_cu_layer[b] + rho]].  Feeds relaxkv_rope. */
+relaxkv_status relaxkv_target_positions(const relaxkv_shape* shape, const int32_t* u_pos, const int32_t* u_cu,
+                                        const int32_t* r_rank, const int32_t* r_cu_layer,
+                                        const int32_t* h_max_targets, int32_t* positions_out, relaxkv_stream stream);
+
+/* Hidden-state carry between layers (Section 3.2: a token stays active through its highest selected layer):
+ * h_out gets, in the row order of layer l+1's targets, the rows of h_in (row order of layer l's targets)
+ * that stay active.  r_cu_layer = r_cu + l*B, r_cu_next = r_cu + (l+1)*B; h_max_next: host bounds on
+ * |R_{l+1,b}|.  h_in, h_out [rows, n_cols], distinct buffers. */
+relaxkv_status relaxkv_carry_rows(const relaxkv_shape* shape, const void* h_in, void* h_out, int32_t n_cols,
+                                  const int32_t* r_rank, const int32_t* r_cu_layer, const int32_t* r_cu_next,
+                                  const int32_t* h_max_next, relaxkv_stream stream);
+
+/*
  * Test utility: the same result as relaxkv_sparse_ctx_attention from a plain SIMT kernel (one warp
  * per output row, fp32 throughout, no tensor cores).  A second opinion for debugging; far slower.
  */

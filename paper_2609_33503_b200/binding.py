@@ -24,7 +24,8 @@ ENTRY_POINTS = (
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_list_attention",
-    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_rope",
+    "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
 
 
@@ -261,6 +262,43 @@ def relaxkv_scatter_kv_lists(shape: Shape, cache: CacheView, k_new: torch.Tensor
 def relaxkv_mean_scores(shape: Shape, n_layers: int, scores: torch.Tensor, mean_out: torch.Tensor, stream=None) -> None:
     _check(lib().relaxkv_mean_scores(shape.ref(), int(n_layers), _ptr(scores), _ptr(mean_out), _stream(stream)),
            "relaxkv_mean_scores")
+
+
+def relaxkv_rmsnorm(x: torch.Tensor, weight: torch.Tensor, y: torch.Tensor, eps: float, stream=None) -> None:
+    _check(lib().relaxkv_rmsnorm(_ptr(x), _ptr(weight), _ptr(y), ctypes.c_int64(x.shape[0]), int(x.shape[1]),
+                                 ctypes.c_float(eps), _stream(stream)), "relaxkv_rmsnorm")
+
+
+def relaxkv_linear(x: torch.Tensor, weight: torch.Tensor, y: torch.Tensor, residual: Optional[torch.Tensor] = None,
+                   stream=None) -> None:
+    """y = x weight^T (+ residual); weight is [n_out, n_in]."""
+    _check(lib().relaxkv_linear(_ptr(x), _ptr(weight), _ptr(residual), _ptr(y), ctypes.c_int64(x.shape[0]),
+                                int(weight.shape[0]), int(weight.shape[1]), _stream(stream)), "relaxkv_linear")
+
+
+def relaxkv_rope(x: torch.Tensor, positions: torch.Tensor, theta: float, stream=None) -> None:
+    """In place on x [rows, heads, D]; positions int32 [rows]."""
+    _check(lib().relaxkv_rope(_ptr(x), ctypes.c_int64(x.shape[0]), int(x.shape[1]), int(x.shape[2]), _ptr(positions),
+                              ctypes.c_float(theta), _stream(stream)), "relaxkv_rope")
+
+
+def relaxkv_swiglu(gate_up: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    _check(lib().relaxkv_swiglu(_ptr(gate_up), _ptr(out), ctypes.c_int64(gate_up.shape[0]), int(out.shape[1]),
+                                _stream(stream)), "relaxkv_swiglu")
+
+
+def relaxkv_target_positions(shape: Shape, u_pos, u_cu, r_rank, r_cu_layer, max_targets: Sequence[int],
+                             positions_out: torch.Tensor, stream=None) -> None:
+    _check(lib().relaxkv_target_positions(shape.ref(), _ptr(u_pos), _ptr(u_cu), _ptr(r_rank), _ptr(r_cu_layer),
+                                          _i32(max_targets), _ptr(positions_out), _stream(stream)),
+           "relaxkv_target_positions")
+
+
+def relaxkv_carry_rows(shape: Shape, h_in: torch.Tensor, h_out: torch.Tensor, r_rank, r_cu_layer, r_cu_next,
+                       max_next: Sequence[int], stream=None) -> None:
+    _check(lib().relaxkv_carry_rows(shape.ref(), _ptr(h_in), _ptr(h_out), int(h_in.shape[1]), _ptr(r_rank),
+                                    _ptr(r_cu_layer), _ptr(r_cu_next), _i32(max_next), _stream(stream)),
+           "relaxkv_carry_rows")
 
 
 def relaxkv_debug_wait_timeout(stream=None) -> None:

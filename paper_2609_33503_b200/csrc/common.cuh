@@ -25,7 +25,7 @@ DeviceStatus* status_word();
 
 enum KernelId : int {
   KID_SETS = 1, KID_SELECT = 2, KID_SCORE = 3, KID_GATHER = 4, KID_SCATTER = 5,
-  KID_ATTN_SIMT = 6, KID_ATTN_SM100 = 7, KID_SCORE_SM100 = 8
+  KID_ATTN_SIMT = 6, KID_ATTN_SM100 = 7, KID_SCORE_SM100 = 8, KID_GEMM_SM100 = 9, KID_DENSE = 10
 };
 
 __device__ __forceinline__ void report(DeviceStatus* st, int status, int kernel, int v0, int v1) {

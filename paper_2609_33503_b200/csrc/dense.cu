@@ -1,0 +1,226 @@
+// The small row-wise kernels of the active targets' block work (Algorithm 1, steps 14, 16, 20): RMSNorm, rotary
+// embedding at the tokens' ORIGINAL positions (Section 3.3), SwiGLU, and the carry of the hidden rows that stay
+// active from layer l to l+1 (R_{l+1} is a subset of R_l).  All HBM-bound, 16-byte accesses.
+#include "common.cuh"
+
+namespace relaxkv {
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(w[e] << 16); f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint32_t w[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+    w[e] = *reinterpret_cast<uint32_t*>(&h2);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// y = x / sqrt(mean(x^2) + eps) * w ; one block per row, C a multiple of 8.
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y, int C, float eps) {
+  const long long row = blockIdx.x;
+  const uint16_t* xr = x + row * C;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 8; i < C; i += 256 * 8) {
+    float f[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(xr + i)), f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+  }
+  __shared__ float red[8];
+  ss = warp_reduce_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];                 // fixed order: reproducible
+  const float inv = rsqrtf(tot / (float)C + eps);
+  for (int i = threadIdx.x * 8; i < C; i += 256 * 8) {
+    float f[8], g[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(xr + i)), f);
+    unpack8(__ldg(reinterpret_cast<const uint4*>(w + i)), g);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = f[e] * inv * g[e];
+    *reinterpret_cast<uint4*>(y + row * C + i) = pack8(f);
+  }
+}
+
+// Rotate-half rotary embedding in place on x [rows, heads, D]; one thread per (row, head, 8 pairs).
+__global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads, int D, const int* __restrict__ positions,
+                            float log2_theta) {
+  const int half = D / 2, groups = half / 8;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * heads * groups) return;
+  const int gi = (int)(idx % groups);
+  const long long rh = idx / groups;
+  const long long row = rh / heads;
+  uint16_t* v = x + rh * D;
+  const double pos = (double)positions[row];
+  float a[8], b[8];
+  unpack8(*reinterpret_cast<const uint4*>(v + gi * 8), a);
+  unpack8(*reinterpret_cast<const uint4*>(v + half + gi * 8), b);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int i = gi * 8 + e;
+    // angle = pos * theta^(-2i/D), reduced in double so that positions of tens of thousands keep their phase
+    const double inv_freq = exp2(-(double)log2_theta * (2.0 * i / D));
+    double ang = pos * inv_freq;
+    ang -= 6.283185307179586 * floor(ang * 0.15915494309189535);
+    float s, c;
+    sincosf((float)ang, &s, &c);
+    const float x1 = a[e], x2 = b[e];
+    a[e] = x1 * c - x2 * s;
+    b[e] = x2 * c + x1 * s;
+  }
+  *reinterpret_cast<uint4*>(v + gi * 8) = pack8(a);
+  *reinterpret_cast<uint4*>(v + half + gi * 8) = pack8(b);
+}
+
+// out[r, i] = silu(gu[r, i]) * gu[r, I + i]
+__global__ void swiglu_kernel(const uint16_t* __restrict__ gu, uint16_t* __restrict__ out, long long rows, int I) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = I / 8;
+  if (idx >= rows * per_row) return;
+  const long long r = idx / per_row;
+  const int i = (int)(idx - r * per_row) * 8;
+  float g[8], u[8];
+  unpack8(__ldg(reinterpret_cast<const uint4*>(gu + r * 2 * I + i)), g);
+  unpack8(__ldg(reinterpret_cast<const uint4*>(gu + r * 2 * I + I + i)), u);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+  *reinterpret_cast<uint4*>(out + r * I + i) = pack8(g);
+}
+
+// positions of the layer's active targets: pos[row] = u_pos[u_cu[b] + r_rank[r_cu[b] + rho]]
+__global__ void target_positions_kernel(ReqTable rt, const int* __restrict__ u_pos, const int* __restrict__ u_cu,
+                                        const int* __restrict__ r_rank, const int* __restrict__ r_cu, int* __restrict__ pos,
+                                        DeviceStatus* st) {
+  const int B = rt.n_req;
+  const int y = blockIdx.x * blockDim.x + threadIdx.x;
+  if (y >= rt.tile_cu[B]) return;
+  const int b = find_segment(rt.tile_cu, B, y);
+  const int rho = y - rt.tile_cu[b];
+  const int nr = r_cu[b + 1] - r_cu[b];
+  if (rho >= nr) return;
+  const int c = r_rank[r_cu[b] + rho];
+  const int nu = u_cu[b + 1] - u_cu[b];
+  if (c < 0 || c >= nu) { report(st, RELAXKV_ERR_BAD_INDEX, KID_DENSE, c, nu); return; }
+  pos[r_cu[b] - r_cu[0] + rho] = u_pos[u_cu[b] + c];
+}
+
+// Hidden rows that stay active: for each target of layer l+1 (rank c), its row among layer l's targets.
+// One block copies one row (C a multiple of 8).
+__global__ void __launch_bounds__(128)
+carry_rows_kernel(ReqTable rt, const uint16_t* __restrict__ h_in, uint16_t* __restrict__ h_out, int C,
+                  const int* __restrict__ r_rank, const int* __restrict__ r_cu_l, const int* __restrict__ r_cu_next,
+                  DeviceStatus* st) {
+  const int B = rt.n_req;
+  __shared__ long long src_row;
+  const int y = blockIdx.x;
+  const int b = find_segment(rt.tile_cu, B, y);
+  const int rho = y - rt.tile_cu[b];
+  const int n_next = r_cu_next[b + 1] - r_cu_next[b];
+  if (rho >= n_next) return;
+  if (threadIdx.x == 0) {
+    const int c = r_rank[r_cu_next[b] + rho];
+    const int* list = r_rank + r_cu_l[b];
+    const int n_l = r_cu_l[b + 1] - r_cu_l[b];
+    int lo = 0, hi = n_l;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (list[mid] < c) lo = mid + 1; else hi = mid; }
+    if (lo >= n_l || list[lo] != c) { report(st, RELAXKV_ERR_BAD_INDEX, KID_DENSE, c, lo); src_row = -1; }
+    else src_row = (long long)(r_cu_l[b] - r_cu_l[0]) + lo;
+  }
+  __syncthreads();
+  if (src_row < 0) return;
+  const long long dst_row = (long long)(r_cu_next[b] - r_cu_next[0]) + rho;
+  for (int i = threadIdx.x * 8; i < C; i += 128 * 8)
+    *reinterpret_cast<uint4*>(h_out + dst_row * C + i) = __ldg(reinterpret_cast<const uint4*>(h_in + src_row * C + i));
+}
+
+}  // namespace relaxkv
+
+using namespace relaxkv;
+
+extern "C" relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64_t n_rows, int32_t n_cols,
+                                          float eps, relaxkv_stream stream) {
+  if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || !(eps >= 0.f)) return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_cols < 8 || (n_cols % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  rmsnorm_kernel<<<(unsigned)n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(y), n_cols, eps);
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
+                                       float theta, relaxkv_stream stream) {
+  if (!x || !positions || !aligned16(x) || !(theta > 1.f)) return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_heads < 1 || (head_dim != 64 && head_dim != 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  const long long n = n_rows * n_heads * (head_dim / 16);
+  rope_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<uint16_t*>(x), n_rows, n_heads, head_dim, positions, log2f(theta));
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t n_rows, int32_t n_inter, relaxkv_stream stream) {
+  if (!gate_up || !out || !aligned16(gate_up) || !aligned16(out)) return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_inter < 8 || (n_inter % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  const long long n = n_rows * (n_inter / 8);
+  swiglu_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint16_t*>(gate_up), static_cast<uint16_t*>(out), n_rows, n_inter);
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_target_positions(const relaxkv_shape* shape, const int32_t* u_pos, const int32_t* u_cu,
+                                                   const int32_t* r_rank, const int32_t* r_cu_layer,
+                                                   const int32_t* h_max_targets, int32_t* positions_out, relaxkv_stream stream) {
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (!u_pos || !u_cu || !r_rank || !r_cu_layer || !h_max_targets || !positions_out) return RELAXKV_ERR_INVALID_ARG;
+  ReqTable rt;
+  fill_req_table(rt, shape, nullptr, nullptr);
+  long long total = 0;
+  for (int b = 0; b < shape->n_req; ++b) {
+    if (h_max_targets[b] < 0) return RELAXKV_ERR_INVALID_ARG;
+    total += h_max_targets[b];
+    rt.tile_cu[b + 1] = (int)total;
+  }
+  if (total == 0) return RELAXKV_OK;
+  if (total > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  target_positions_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      rt, u_pos, u_cu, r_rank, r_cu_layer, positions_out, st);
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_carry_rows(const relaxkv_shape* shape, const void* h_in, void* h_out, int32_t n_cols,
+                                             const int32_t* r_rank, const int32_t* r_cu_layer, const int32_t* r_cu_next,
+                                             const int32_t* h_max_next, relaxkv_stream stream) {
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (!h_in || !h_out || !r_rank || !r_cu_layer || !r_cu_next || !h_max_next || !aligned16(h_in) || !aligned16(h_out))
+    return RELAXKV_ERR_INVALID_ARG;
+  if (n_cols < 8 || (n_cols % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  ReqTable rt;
+  fill_req_table(rt, shape, nullptr, nullptr);
+  long long total = 0;
+  for (int b = 0; b < shape->n_req; ++b) {
+    if (h_max_next[b] < 0) return RELAXKV_ERR_INVALID_ARG;
+    total += h_max_next[b];
+    rt.tile_cu[b + 1] = (int)total;
+  }
+  if (total == 0) return RELAXKV_OK;
+  if (total > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  carry_rows_kernel<<<(unsigned)total, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      rt, static_cast<const uint16_t*>(h_in), static_cast<uint16_t*>(h_out), n_cols, r_rank, r_cu_layer, r_cu_next, st);
+  return launch_ok();
+}

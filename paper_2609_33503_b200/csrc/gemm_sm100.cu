@@ -1,0 +1,163 @@
+// y = x W^T (+ residual) on the Blackwell tensor cores: the projections of the active targets' block work
+// (Algorithm 1, steps 16 and 20).  x [M, K], W [N, K] (the [out, in] layout), y [M, N], bf16 with fp32
+// accumulation in TMEM.  CTA tile 128 x 256, K blocks of 64 through a 4-stage TMA ring (128-byte swizzle),
+// one MMA issuer thread (tcgen05.mma M=128, N=256, K=16), four epilogue warps (thread = row = TMEM lane).
+// Tiles are walked in groups of 16 row tiles so that a wave's working set (x rows + W rows) stays in L2.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace relaxkv {
+
+using namespace ptx;
+
+bool make_map_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                 uint64_t stride2_bytes, uint32_t b1, uint32_t b2);          // attention_sm100.cu
+
+constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64, kGemmStages = 4, kGemmThreads = 192, kGemmGroupM = 16;
+constexpr int kGemmABytes = kGemmBM * kGemmBK * 2, kGemmBBytes = kGemmBN * kGemmBK * 2;
+constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 8 * (2 * kGemmStages + 1) + 16 + 1024;
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                  long long M, int N, int K, uint16_t* __restrict__ y, const uint16_t* __restrict__ residual,
+                  DeviceStatus* st) {
+  // ---- which tile (grouped order: kGemmGroupM row tiles x all column tiles at a time) ----
+  const int tiles_m = (int)((M + kGemmBM - 1) / kGemmBM), tiles_n = (N + kGemmBN - 1) / kGemmBN;
+  const int pid = blockIdx.x;
+  const int per_group = kGemmGroupM * tiles_n;
+  const int group = pid / per_group, first_m = group * kGemmGroupM;
+  const int group_m = min(tiles_m - first_m, kGemmGroupM);
+  const int tm = first_m + (pid % per_group) % group_m, tn = (pid % per_group) / group_m;
+  if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar0 = base + kGemmStages * kGemmStageBytes;
+  const uint32_t bar_full = bar0, bar_empty = bar0 + 8 * kGemmStages, bar_acc = bar0 + 16 * kGemmStages;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kGemmStages * kGemmStageBytes + 8 * (2 * kGemmStages + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(const_cast<uint32_t*>(tmem_slot) + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGemmStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_acc, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 5) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_k = (K + kGemmBK - 1) / kGemmBK;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      prefetch_tensormap(&tm_a); prefetch_tensormap(&tm_b);
+      for (int kt = 0; kt < n_k; ++kt) {
+        const int s = kt % kGemmStages;
+        if (kt >= kGemmStages && !mbar_wait(bar_empty + 8 * s, ((kt / kGemmStages) - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(bar_full + 8 * s, kGemmStageBytes);
+        tma_load_3d(base + s * kGemmStageBytes, &tm_a, bar_full + 8 * s, kt * kGemmBK, tm * kGemmBM, 0);
+        tma_load_3d(base + s * kGemmStageBytes + kGemmABytes, &tm_b, bar_full + 8 * s, kt * kGemmBK, tn * kGemmBN, 0);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16_f32(kGemmBM, kGemmBN, 0);
+      bool ok = true;
+      for (int kt = 0; kt < n_k; ++kt) {
+        const int s = kt % kGemmStages;
+        if (!(ok = mbar_wait(bar_full + 8 * s, (kt / kGemmStages) & 1, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t a = base + s * kGemmStageBytes;
+        mma_ss_4steps(tmem_base, desc_lo(a, 16), desc_lo(a + kGemmABytes, 16), desc_hi_sw128(1024), idesc, kt > 0 ? 1u : 0u);
+        mma_commit(bar_empty + 8 * s);
+      }
+      if (ok) mma_commit(bar_acc);
+    }
+  } else {
+    // ---- epilogue: thread = output row = TMEM lane ----
+    bool ok = mbar_wait(bar_acc, 0, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const long long row = (long long)tm * kGemmBM + warp * 32 + lane;
+      const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kGemmBN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + c * 32, v);
+        tmem_wait_ld();
+        const int col0 = tn * kGemmBN + c * 32;
+        if (row < M && col0 < N) {
+          const long long off = row * N + col0;
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            if (col0 + i < N) {                                  // N is a multiple of 8
+              float f[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i + e]);
+              if (residual != nullptr) {
+                const uint4 r = __ldg(reinterpret_cast<const uint4*>(residual + off + i));
+                const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { f[2 * e] += __uint_as_float(rw[e] << 16); f[2 * e + 1] += __uint_as_float(rw[e] & 0xffff0000u); }
+              }
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+                w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(y + off + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_GEMM_SM100, tm, tn);
+    const uint64_t tw = global_timer_ns();
+    while (global_timer_ns() - tw < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, 256); }
+}
+
+}  // namespace relaxkv
+
+using namespace relaxkv;
+
+extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
+                                         int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream_) {
+  if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || (residual && !aligned16(residual)))
+    return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_out < 8 || n_in < 8 || (n_out % 8) || (n_in % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  CUtensorMap tm_a, tm_b;
+  if (!make_map_3d(&tm_a, x, (uint64_t)n_in, (uint64_t)n_rows, 1, (uint64_t)n_in * 2, (uint64_t)n_in * 2 * (uint64_t)n_rows, kGemmBM, 1) ||
+      !make_map_3d(&tm_b, weight, (uint64_t)n_in, (uint64_t)n_out, 1, (uint64_t)n_in * 2, (uint64_t)n_in * 2 * (uint64_t)n_out, kGemmBN, 1))
+    return RELAXKV_ERR_CUDA;
+  DeviceStatus* st = status_word();
+  if (!st) return RELAXKV_ERR_CUDA;
+  static bool attr_done[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(gemm_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess)
+      return RELAXKV_ERR_CUDA;
+    attr_done[dev] = true;
+  }
+  const long long tiles_m = (n_rows + kGemmBM - 1) / kGemmBM, tiles_n = (n_out + kGemmBN - 1) / kGemmBN;
+  if (tiles_m * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  gemm_sm100_kernel<<<(unsigned)(tiles_m * tiles_n), kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
+      tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), st);
+  return launch_ok();
+}

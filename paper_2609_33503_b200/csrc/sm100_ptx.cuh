@@ -192,6 +192,17 @@ __device__ __forceinline__ void mma_ss_kloop(uint32_t d_tmem, uint32_t a_lo, uin
   }
 }
 
+// D[tmem] (+)= A[smem] * B[smem] for four K steps of 16 inside one 64-element (128-byte) swizzled K block.
+// acc_first = 0 makes the first MMA overwrite D.
+__device__ __forceinline__ void mma_ss_4steps(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                              uint32_t acc_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      RELAXKV_MMA_SS_STEP(0, p0) RELAXKV_MMA_SS_STEP(2, p1) RELAXKV_MMA_SS_STEP(4, p1) RELAXKV_MMA_SS_STEP(6, p1)
+      "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first) : "memory");
+}
+
 #define RELAXKV_MMA_TS_STEP(AOFF, BOFF, PRED)                                                  \
   "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                                  \
   "mov.b64 db, {tb, %3};\n\t"                                                                  \
