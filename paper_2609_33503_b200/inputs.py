@@ -214,3 +214,44 @@ NAMED: Dict[str, object] = {
     "qwen14b_32k": qwen14b_32k,
     "ragged8": ragged8,
 }
+
+
+# ----------------------------------------------------------------------------
+# Synthetic decoder-block weights (the paper's models are not here)
+# ----------------------------------------------------------------------------
+
+@dataclasses.dataclass(frozen=True)
+class BlockShape:
+    """Llama-style pre-norm decoder block: hidden size, SwiGLU width, rotary base, RMSNorm epsilon."""
+    hidden: int
+    inter: int
+    rope_theta: float = 1.0e6
+    eps: float = 1.0e-6
+
+
+QWEN3_14B_BLOCK = BlockShape(hidden=5120, inter=17408)
+LLAMA31_8B_BLOCK = BlockShape(hidden=4096, inter=14336, rope_theta=5.0e5, eps=1.0e-5)
+
+
+def block_weights(w: Workload, blk: BlockShape, layer: int, device="cpu") -> Dict[str, torch.Tensor]:
+    """Random-init weights of one block, bf16: projections ~ N(0, 1/fan_in) in the [out, in] layout, norm gains
+    ~ 1 + 0.1 N(0,1).  `w_gate_up` stacks the gate rows on top of the up rows."""
+    g = _gen(device, 7_000_000 + w.base_seed + layer)
+    C, H, Hkv, D, I = blk.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, blk.inter
+
+    def lin(n_out, n_in):
+        return (torch.randn(n_out, n_in, generator=g, device=device, dtype=torch.float32) * n_in ** -0.5).to(torch.bfloat16)
+
+    def gain(n):
+        return (1.0 + 0.1 * torch.randn(n, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
+
+    return {"w_in_norm": gain(C), "wq": lin(H * D, C), "wk": lin(Hkv * D, C), "wv": lin(Hkv * D, C), "wo": lin(C, H * D),
+            "w_post_norm": gain(C), "w_gate_up": lin(2 * I, C), "w_down": lin(C, I)}
+
+
+def input_representations(w: Workload, blk: BlockShape, req: int, positions: torch.Tensor, device="cpu") -> torch.Tensor:
+    """Stand-in for the input embeddings of the tokens at `positions` (Algorithm 1, step 14): N(0,1) rows,
+    a pure function of (request, position)."""
+    g = _gen(device, 9_000_000 + w.base_seed + req)
+    table = torch.randn(w.ctx_lens[req], blk.hidden, generator=g, device=device, dtype=torch.float32)
+    return table[positions.to(device=device, dtype=torch.long)].to(torch.bfloat16)

@@ -93,3 +93,77 @@ def test_target_positions_and_row_carry():
             np.testing.assert_array_equal(out.float().cpu().numpy().astype(np.float64), np.concatenate(refs))
     st, detail = B().relaxkv_read_device_status()
     assert st == 0, (st, detail)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round float64 values to bf16 (nearest even) and return them as float64 - the storage precision of
+    every tensor that travels between two kernels."""
+    t = torch.from_numpy(np.ascontiguousarray(x)).to(torch.float32).to(torch.bfloat16)
+    return t.to(torch.float64).numpy()
+
+
+def to_bits(x: np.ndarray) -> np.ndarray:
+    return inputs.bf16_bits(torch.from_numpy(np.ascontiguousarray(x)).to(torch.float32).to(torch.bfloat16))
+
+
+def test_whole_repair_loop_with_block_work():
+    """Algorithm 1, steps 13-22, three layers: the CUDA layer loop against the oracle chain.  The reference
+    rounds every tensor that the GPU stores in bf16 to bf16 at the same points (storage precision is part of
+    the data path); inside an operation it stays fp64."""
+    from paper_2609_33503_b200.layer_loop import LayerLoop
+    from tests.harness import Case
+    w = inputs.Workload("block", 3, 4, 2, 64, 64, (600, 380), (8, 5), 0.15, base_seed=3,
+                        planted_chunks=((2, 7), (1,)), variant="calibrated")
+    blkshape = inputs.BlockShape(hidden=256, inter=512, rope_theta=1.0e4, eps=1.0e-5)
+    case = Case(w)
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    n_u, n_r = s.counts()
+    weights = [inputs.block_weights(w, blkshape, l, "cuda") for l in range(w.n_layers)]
+    h0 = torch.cat([inputs.input_representations(w, blkshape, b, torch.from_numpy(case.sets[b].u_pos.astype(np.int64)), "cuda")
+                    for b in range(w.n_req)]).contiguous()
+    k_gpu = [k.clone() for k in case.k_cache]
+    v_gpu = [v.clone() for v in case.v_cache]
+    views = [B().CacheView(k, v, [int(x) for x in case.ctx_cu[:-1]]) for k, v in zip(k_gpu, v_gpu)]
+    loop = LayerLoop(s, blkshape, sum(n_u))
+    h_gpu = loop.run(h0, weights, views)
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+
+    # ---- oracle chain, request by request ----
+    H, Hkv, D = w.n_q_heads, w.n_kv_heads, w.head_dim
+    off_u, final_refs = 0, []
+    for b in range(w.n_req):
+        sets = case.sets[b]
+        h = blk.f64(bits(h0[off_u:off_u + len(sets.u_pos)]))
+        off_u += len(sets.u_pos)
+        for l in range(w.n_layers):
+            W = {k_: blk.f64(bits(v_)) for k_, v_ in weights[l].items()}
+            pos = sets.positions(l)
+            n = len(pos)
+            x = bf16_round(blk.rmsnorm(h, W["w_in_norm"], blkshape.eps))
+            q = bf16_round(blk.linear(x, W["wq"])).reshape(n, H, D)
+            k = bf16_round(blk.linear(x, W["wk"])).reshape(n, Hkv, D)
+            v = bf16_round(blk.linear(x, W["wv"])).reshape(n, Hkv, D)
+            q, k = bf16_round(blk.rope(q, pos, blkshape.rope_theta)), bf16_round(blk.rope(k, pos, blkshape.rope_theta))
+            o, _ = orc.repair_attention(case.req_k(l, b), case.req_v(l, b), to_bits(q), to_bits(k), to_bits(v), sets.u_pos,
+                                        sets.ranks(l), case.scale)
+            o = bf16_round(o).reshape(n, H * D)
+            # cache update: the GPU's repaired cache rows hold (its own) k, v of this layer
+            lo = int(case.ctx_cu[b])
+            gk = k_gpu[l][lo + torch.from_numpy(pos.astype(np.int64)).cuda()].float().cpu().numpy()
+            dk = np.abs(gk - k)          # single-ulp differences of earlier tensors propagate: ~1 % of |k| on average
+            assert dk.max() <= 0.1 * max(1.0, np.abs(k).max()) and dk.mean() <= 1e-2 * np.abs(k).mean(), (l, dk.max(), dk.mean())
+            a = bf16_round(blk.linear(o, W["wo"], h))
+            x2 = bf16_round(blk.rmsnorm(a, W["w_post_norm"], blkshape.eps))
+            m = bf16_round(blk.swiglu(bf16_round(blk.linear(x2, W["w_gate_up"]))))
+            h_out = bf16_round(blk.linear(m, W["w_down"], a))
+            h = blk.compact_rows(h_out, sets.ranks(l), sets.ranks(l + 1)) if l + 1 < w.n_layers else h_out
+        final_refs.append(h)
+    ref = np.concatenate(final_refs)
+    got = h_gpu.float().cpu().numpy().astype(np.float64)
+    assert got.shape == ref.shape
+    err = np.abs(got - ref)
+    scale_ = np.abs(ref).mean()
+    # three layers of bf16 tensors: single-ulp differences (fp32 vs fp64 accumulation) propagate, nothing more
+    assert err.mean() <= 1e-2 * scale_ and err.max() <= 0.15 * max(1.0, np.abs(ref).max()), (err.mean(), err.max(), scale_)
