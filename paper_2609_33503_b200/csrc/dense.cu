@@ -50,20 +50,17 @@ rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, u
   }
 }
 
-// Rotate-half rotary embedding in place on x [rows, heads, D]; one thread per (row, head, 8 pairs).
+// Rotate-half rotary embedding in place on x [rows, heads, D]; one thread per (row, 8 pairs): the eight
+// (cos, sin) pairs are computed once and applied to every head of the row.
 __global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads, int D, const int* __restrict__ positions,
                             float log2_theta) {
   const int half = D / 2, groups = half / 8;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * heads * groups) return;
+  if (idx >= rows * groups) return;
   const int gi = (int)(idx % groups);
-  const long long rh = idx / groups;
-  const long long row = rh / heads;
-  uint16_t* v = x + rh * D;
+  const long long row = idx / groups;
   const double pos = (double)positions[row];
-  float a[8], b[8];
-  unpack8(*reinterpret_cast<const uint4*>(v + gi * 8), a);
-  unpack8(*reinterpret_cast<const uint4*>(v + half + gi * 8), b);
+  float cs[8], sn[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     const int i = gi * 8 + e;
@@ -71,14 +68,22 @@ __global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads,
     const double inv_freq = exp2(-(double)log2_theta * (2.0 * i / D));
     double ang = pos * inv_freq;
     ang -= 6.283185307179586 * floor(ang * 0.15915494309189535);
-    float s, c;
-    sincosf((float)ang, &s, &c);
-    const float x1 = a[e], x2 = b[e];
-    a[e] = x1 * c - x2 * s;
-    b[e] = x2 * c + x1 * s;
+    sincosf((float)ang, &sn[e], &cs[e]);
   }
-  *reinterpret_cast<uint4*>(v + gi * 8) = pack8(a);
-  *reinterpret_cast<uint4*>(v + half + gi * 8) = pack8(b);
+  for (int h = 0; h < heads; ++h) {
+    uint16_t* v = x + (row * heads + h) * D;
+    float a[8], b[8];
+    unpack8(*reinterpret_cast<const uint4*>(v + gi * 8), a);
+    unpack8(*reinterpret_cast<const uint4*>(v + half + gi * 8), b);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float x1 = a[e], x2 = b[e];
+      a[e] = x1 * cs[e] - x2 * sn[e];
+      b[e] = x2 * cs[e] + x1 * sn[e];
+    }
+    *reinterpret_cast<uint4*>(v + gi * 8) = pack8(a);
+    *reinterpret_cast<uint4*>(v + half + gi * 8) = pack8(b);
+  }
 }
 
 // out[r, i] = silu(gu[r, i]) * gu[r, I + i]
@@ -161,7 +166,7 @@ extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads,
   if (!x || !positions || !aligned16(x) || !(theta > 1.f)) return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_heads < 1 || (head_dim != 64 && head_dim != 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
-  const long long n = n_rows * n_heads * (head_dim / 16);
+  const long long n = n_rows * (head_dim / 16);
   rope_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<uint16_t*>(x), n_rows, n_heads, head_dim, positions, log2f(theta));
   return launch_ok();
