@@ -297,7 +297,10 @@ relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* res
 
 /* Rotary embedding in place, rotate-half convention: pair i < D/2 of each head vector is rotated by
  * positions[row] * theta^(-2i/D).  x [n_rows, n_heads, head_dim]; positions: device int32 [n_rows], the rows'
- * ORIGINAL global positions (Section 3.3: restricting the context does not renumber tokens). */
+ * ORIGINAL global positions (Section 3.3: restricting the context does not renumber tokens).  Rotations
+ * compose, so the same call re-aligns the cached keys of a chunk that is placed at another offset than the
+ * one it was encoded at (Section 2, positional consistency): pass the offset difference (it may be negative)
+ * as every token's position. */
 relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
                             float theta, relaxkv_stream stream);
 

@@ -167,3 +167,31 @@ def test_whole_repair_loop_with_block_work():
     scale_ = np.abs(ref).mean()
     # three layers of bf16 tensors: single-ulp differences (fp32 vs fp64 accumulation) propagate, nothing more
     assert err.mean() <= 1e-2 * scale_ and err.max() <= 0.15 * max(1.0, np.abs(ref).max()), (err.mean(), err.max(), scale_)
+
+
+def test_rope_realigns_keys_of_a_moved_chunk():
+    """Positional consistency (Section 2): a chunk cached at one offset and placed at another is re-aligned by
+    rotating its cached keys by the offset difference.  The keys of a 512-token chunk are rotated at offset
+    4096, then shifted by +8192 and by -3072 with the same kernel (positions = the delta for every token);
+    the result must equal the oracle's rotation at the final positions."""
+    T, Hkv, D, theta = 512, 8, 128, 1.0e6
+    k_raw = rnd(T, Hkv, D, seed=21)
+    old = torch.arange(4096, 4096 + T, dtype=torch.int32, device="cuda")
+    for delta in (8192, -3072):
+        k = k_raw.clone()
+        B().relaxkv_rope(k, old, theta)                                               # the cached, chunk-time rotation
+        B().relaxkv_rope(k, torch.full((T,), delta, dtype=torch.int32, device="cuda"), theta)   # re-alignment
+        ref = blk.rope(blk.f64(bits(k_raw)), (old.cpu().numpy().astype(np.int64) + delta), theta)
+        # two bf16 roundings instead of one
+        g = k.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(g - ref) <= 2.0 ** -7 * np.abs(ref) + 2e-2), float(np.abs(g - ref).max())
+        # and attention logits against a query at a fixed position keep their relative-offset meaning
+        q = rnd(1, Hkv, D, seed=22)
+        qpos = torch.tensor([4096 + delta + T], dtype=torch.int32, device="cuda")
+        B().relaxkv_rope(q, qpos, theta)
+        logits = (q.float()[0][None] * k.float()).sum(-1).cpu().numpy()               # [T, Hkv]
+        q_ref = blk.rope(blk.f64(bits(rnd(1, Hkv, D, seed=22))), qpos.cpu().numpy(), theta)
+        ref_logits = (q_ref[0][None] * ref).sum(-1)
+        assert np.abs(logits - ref_logits).max() <= 0.02 * np.sqrt(D) + 0.05 * np.abs(ref_logits).max()
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (st, detail)
