@@ -472,8 +472,14 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
   auto kern = attention_sm100_kernel<D>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess)
-    return RELAXKV_ERR_CUDA;
+  static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess)
+      return RELAXKV_ERR_CUDA;
+    attr_done[dev] = true;
+  }
   kern<<<(unsigned)grid, kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
       tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
       r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, st);
