@@ -46,7 +46,7 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
-                       int mode, int allow_empty, int H, int Hkv, int tile_targets, float scale_log2,
+                       int mode, int allow_empty, int head_inner, int H, int Hkv, int tile_targets, float scale_log2,
                        const int* __restrict__ u_pos, const int* __restrict__ u_cu,
                        const int* __restrict__ r_rank, const int* __restrict__ r_cu,
                        long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
@@ -61,8 +61,10 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int B = rt.n_req;
   const int G = H / Hkv;
   const int n_pairs_total = rt.tile_cu[B];
-  const int hd = blockIdx.x / n_pairs_total;                  // KV head outermost: its K/V stays in L2
-  const int tt = blockIdx.x - hd * n_pairs_total;
+  // Block order.  Large contexts: KV head outermost, so one head's K/V stays in L2 while its tiles run.
+  // Contexts that fit L2 whole (head_inner): tile pair outermost, so the longest tiles of every head start first.
+  const int hd = head_inner ? (int)(blockIdx.x % Hkv) : (int)(blockIdx.x / n_pairs_total);
+  const int tt = head_inner ? (int)(blockIdx.x / Hkv) : (int)(blockIdx.x - hd * n_pairs_total);
   const int b = find_segment(rt.tile_cu, B, tt);
   const int p_rev = tt - rt.tile_cu[b];
   const int nr = r_cu[b + 1] - r_cu[b];
@@ -471,6 +473,10 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
     return RELAXKV_ERR_CUDA;
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
+  // the materialised context (K and V, all heads) against the 126 MB L2
+  long long ctx_rows_used = 0;
+  for (int b = 0; b < B; ++b) ctx_rows_used += plan.rt.bound_b[b];
+  const int head_inner = (ctx_rows_used * (long long)row_kv * 2 <= (40ll << 20)) ? 1 : 0;
   auto kern = attention_sm100_kernel<D>;
   static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
   int dev = 0;
@@ -481,7 +487,7 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
     attr_done[dev] = true;
   }
   kern<<<(unsigned)grid, kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
-      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
+      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
       r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, st);
   return launch_ok();
 }
