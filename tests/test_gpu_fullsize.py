@@ -70,3 +70,92 @@ def test_llama8b_16k_full_size():
 
 def test_qwen14b_32k_full_context_two_layers():
     run_full(inputs.qwen14b_32k("calibrated", 0.15, n_layers=2), tile_targets=25, n_spread=24)
+
+
+def test_maximum_batch_of_64_requests():
+    """The request table's limit (64 requests in one call) with ragged lengths from 1 token upwards:
+    scores, anchors, sets, attention of every row, and the cache update against the oracle."""
+    from paper_2609_33503_b200 import binding as B
+    rng = np.random.default_rng(64)
+    ctx = tuple(int(x) for x in np.concatenate([[1, 2, 127, 128, 129, 700], rng.integers(3, 600, size=58)]))
+    q = tuple(int(x) for x in rng.integers(1, 40, size=64))
+    w = inputs.scaled_down(inputs.qwen14b_32k("literal"), ctx, q, n_layers=2, chunk=64).replace(ratio=0.2)
+    assert w.n_req == 64
+    case = Case(w)
+    s = case.make_session()
+    views = case.cache_views()
+    s.score_select(case.q_layers, views)
+    anchors = s.anchors.cpu().numpy()
+    for l in range(w.n_layers):
+        for b in range(w.n_req):
+            check_anchor_band(case.raw[(l, b)], case.k[b], anchors[l, case.k_cu[b]:case.k_cu[b + 1]])
+    s.build_active_sets(case.anchors_tensor())
+    n_u, n_r = s.counts()
+    assert n_u == [len(case.sets[b].u_pos) for b in range(64)]
+    u_pos, u_cu = s.u_pos.cpu().numpy(), s.u_cu.cpu().numpy()
+    for b in range(64):
+        assert np.array_equal(u_pos[u_cu[b]:u_cu[b + 1]], case.sets[b].u_pos)
+    for l in range(w.n_layers):
+        assert n_r[l] == case.max_targets(l)
+        f = case.fresh[l]
+        out = torch.zeros_like(f.q_new)
+        s.attention(l, views[l], f.q_new, f.k_new, f.v_new, out, case.max_targets(l), case.max_ctx())
+        st, detail = B.relaxkv_read_device_status()
+        assert st == 0, (st, detail)
+        for b in range(64):
+            ref, _ = case.oracle_attention(l, b)
+            mx, mean = attention_errors(out[f.row_cu[b]:f.row_cu[b + 1]], ref)
+            assert mx <= MAX_ABS and mean <= MEAN_ABS, (l, b, mx, mean)
+        k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+        s.scatter(l, B.CacheView(k2, v2, [int(x) for x in case.ctx_cu[:-1]]), f.k_new, f.v_new, case.max_targets(l))
+        for b in range(64):
+            pos = torch.from_numpy(case.sets[b].positions(l).astype(np.int64)).to(k2.device) + int(case.ctx_cu[b])
+            assert torch.equal(k2[pos], f.k_new[f.row_cu[b]:f.row_cu[b + 1]])
+        assert int((k2 != case.k_cache[l]).any(dim=(1, 2)).sum()) <= sum(case.max_targets(l))
+    # one request more than the table holds is refused before any launch
+    too_many = B.Shape(w.n_q_heads, w.n_kv_heads, w.head_dim, ctx + (5,), q + (1,))
+    assert B.relaxkv_workspace_bytes(too_many, 2, case.k + [1]) == 0
+
+
+def test_ragged_batch_with_a_64k_context_sampled_rows():
+    """Two requests of the ragged benchmark batch (65 536 and 8 192 context tokens) in one call, two layers,
+    Qwen3-14B head geometry.  The anchors are drawn at random (the oracle's scoring of 64K keys is not needed
+    to check what follows): the repair schedule must match the oracle's bit for bit, the attention of
+    sampled target rows and the cache update must match the oracle."""
+    from paper_2609_33503_b200 import binding as B
+    ctx, q = (65536, 8192), (64, 32)
+    w = inputs.scaled_down(inputs.qwen14b_32k("calibrated"), ctx, q, n_layers=2, chunk=512)
+    rng = np.random.default_rng(7)
+    k = [max(1, round(0.15 * t)) for t in ctx]
+    override = [[np.sort(rng.choice(t, size=kb, replace=False)).astype(np.int32) for t, kb in zip(ctx, k)] for _ in range(2)]
+    case = Case(w, anchors_override=override)
+    assert case.k == k
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    n_u, n_r = s.counts()
+    u_pos, u_cu = s.u_pos.cpu().numpy(), s.u_cu.cpu().numpy()
+    r_rank, r_cu = s.r_rank.cpu().numpy(), s.r_cu.cpu().numpy()
+    for b in range(2):
+        assert np.array_equal(u_pos[u_cu[b]:u_cu[b + 1]], case.sets[b].u_pos)
+    views = case.cache_views()
+    for l in range(2):
+        for b in range(2):
+            i = l * 2 + b
+            assert np.array_equal(r_rank[r_cu[i]:r_cu[i + 1]], case.sets[b].ranks(l))
+        f = case.fresh[l]
+        out = torch.zeros_like(f.q_new)
+        s.attention(l, views[l], f.q_new, f.k_new, f.v_new, out, n_r[l], n_u)
+        st, detail = B.relaxkv_read_device_status()
+        assert st == 0, (st, detail)
+        for b in range(2):
+            n = f.row_cu[b + 1] - f.row_cu[b]
+            rows = sampled_rows(n, 50, 12, seed=10 * l + b)
+            ref, _ = case.oracle_attention(l, b, rows=rows)
+            got = out[f.row_cu[b]:f.row_cu[b + 1]][torch.from_numpy(rows.astype(np.int64)).to(out.device)]
+            mx, mean = attention_errors(got, ref)
+            assert mx <= MAX_ABS and mean <= MEAN_ABS, (l, b, mx, mean)
+        k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+        s.scatter(l, B.CacheView(k2, v2, [0, ctx[0]]), f.k_new, f.v_new, n_r[l])
+        for b in range(2):
+            pos = torch.from_numpy(case.sets[b].positions(l).astype(np.int64)).to(k2.device) + (0 if b == 0 else ctx[0])
+            assert torch.equal(k2[pos], f.k_new[f.row_cu[b]:f.row_cu[b + 1]]) and torch.equal(v2[pos], f.v_new[f.row_cu[b]:f.row_cu[b + 1]])
