@@ -294,19 +294,27 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
       }
       float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
+      const float neg_m = -m;
 #pragma unroll
       for (int c = 0; c < kBN / 32; ++c) {
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i]), scale_log2, -m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 1]), scale_log2, -m));
-          const float p2 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 2]), scale_log2, -m));
-          const float p3 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + i + 3]), scale_log2, -m));
-          zs0 += p0; zs1 += p1; zs2 += p2; zs3 += p3;
-          __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
-          pk[i >> 1] = *reinterpret_cast<uint32_t*>(&h01);
-          pk[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h23);
+        for (int i = 0; i < 32; i += 8) {
+          // p = 2^(s * scale - m) for eight keys; the scaling and the row sums use packed fp32 pairs
+          float x[8], p[8];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2)
+            fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
+                 scale_log2, neg_m, neg_m);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
+          add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
+          add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(p[e], p[e + 1]);
+            pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h);
+          }
         }
         tmem_st16(t_s + c * 16, pk);
         if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
