@@ -365,6 +365,63 @@ def run_e2e(job, args, mode, world):
             "steps": n, "how": "pinned host buffers, 3 streams (copy-in | kernels | copy-out), 3 layers in flight"}
 
 
+def run_query_attention(args):
+    """Attention of the user query over the (repaired) context cache with the same kernel, through
+    relaxkv_list_attention: the query's prefill rows (the workload's Q rows, every context position visible)
+    and a one-token decode step.  Few query tiles, so the kernel splits each tile's context over several
+    blocks; `unsplit_us` is the same call with the split switched off."""
+    from paper_2609_33503_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = make_workload(args)
+    H, Hkv, D, T = w.n_q_heads, w.n_kv_heads, w.head_dim, w.ctx_lens[0]
+    _, k, v = inputs.layer_qkv(w, 0, 0, dev)
+    view = B.CacheView(k.contiguous(), v.contiguous(), [0])
+    out = {"metric": "query_attention_us", "unit": "us", "higher_is_better": False, "n_gpus": 1, "steps": args.steps,
+           "warmup": args.warmup, "data": "synthetic", "dtype": "bf16",
+           "config": {"workload": w.name, "heads": f"{H}/{Hkv}", "head_dim": D, "ctx_len": T}}
+    for name, Q in (("prefill", w.q_lens[0]), ("decode", 1)):
+        shape = B.Shape(H, Hkv, D, [T], [Q])
+        g = torch.Generator(device=dev).manual_seed(11)
+        q = torch.randn(Q, H, D, device=dev, generator=g).to(torch.bfloat16)
+        o = torch.empty_like(q)
+        ctx_pos = torch.arange(T, dtype=torch.int32, device=dev)
+        ctx_cu = torch.tensor([0, T], dtype=torch.int32, device=dev)
+        tgt_pos = torch.arange(T - Q, T, dtype=torch.int32, device=dev)
+        tgt_cu = torch.tensor([0, Q], dtype=torch.int32, device=dev)
+        nbytes = B.relaxkv_workspace_bytes(shape, 1, [1])
+        ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
+        off = (-ws.data_ptr()) % 256
+        ws = ws[off:off + nbytes]
+        res = {}
+        for label, forced in (("unsplit_us", 1), ("us", 0)):
+            B.relaxkv_debug_set_attention_splits(forced)
+            try:
+                def call():
+                    B.relaxkv_list_attention(shape, view, q, None, None, ctx_pos, ctx_cu, tgt_pos, tgt_cu, [Q], [T], o, ws)
+                for _ in range(max(3, args.warmup)):
+                    call()
+                torch.cuda.synchronize()
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                n = max(10, args.steps)
+                a.record()
+                for _ in range(n):
+                    call()
+                b_.record()
+                torch.cuda.synchronize()
+                res[label] = round(a.elapsed_time(b_) / n * 1e3, 1)
+            finally:
+                B.relaxkv_debug_set_attention_splits(0)
+        res["rows"] = Q
+        res["kv_bytes"] = 2 * T * Hkv * D * 2
+        out[name] = res
+    st, detail = B.relaxkv_read_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {B.status_string(st)} {detail}")
+    out["value"] = out["prefill"]["us"]
+    print(json.dumps(out))
+
+
 def run_dense(args):
     """The whole repair loop (selection, schedule, then per layer: block work of the active rows + repair
     attention + cache update) on one GPU with synthetic block weights of the workload's model family."""
@@ -569,12 +626,16 @@ def main():
     ap.add_argument("--dense", action="store_true",
                     help="run the whole repair loop of Algorithm 1 including the active rows' block work (projections, "
                          "rotary embedding, MLP with synthetic weights); prints its own JSON line")
+    ap.add_argument("--query-attention", action="store_true",
+                    help="time the user query's prefill rows and a decode step over the context cache (same kernel, context split)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows", type=int, default=256)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.query_attention:
+        run_query_attention(args)
     elif args.dense:
         run_dense(args)
     else:

@@ -334,6 +334,15 @@ relaxkv_status relaxkv_sparse_ctx_attention_simt(
     void* workspace, size_t workspace_bytes, relaxkv_stream stream);
 
 /*
+ * Test utility (the paper has no counterpart).  The attention calls split every query tile's context over
+ * several thread blocks when there are too few query tiles to fill the GPU (a query prefill, a decode step, a
+ * layer with few active targets) and merge the partial results by their log-sum-exp; the split count is
+ * chosen from the launch size.  n_splits > 0 forces that count (up to 32, and as far as the workspace's
+ * 2048 row-splits allow) for every later call of this process, 0 restores the automatic choice.
+ */
+relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits);
+
+/*
  * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on
  * a barrier nothing will ever complete.  The wait gives up after its limit (0.4 s), the kernel ends
  * normally and RELAXKV_ERR_TIMEOUT is recorded in the device status word - the same path a stuck

@@ -11,6 +11,8 @@ struct AttnPlan {
   uint16_t* vctx;
   long long ctx_rows;     // rows the two buffers hold (tensor-map extent)
   long long sum_targets;  // sum of the host bounds on |R_{l,b}|
+  float* split_o;         // workspace for a context split across blocks: [kSplitRowsCap, H, D] and [kSplitRowsCap, H]
+  float* split_lse;
 };
 
 // Validates the arguments of an attention call and enqueues the gather of the mixed context into
@@ -53,6 +55,8 @@ inline relaxkv_status prepare_attention(
   plan.kctx = reinterpret_cast<uint16_t*>(base + ws.kctx);
   plan.vctx = reinterpret_cast<uint16_t*>(base + ws.vctx);
   plan.ctx_rows = ws.ctx_rows_cap;
+  plan.split_o = reinterpret_cast<float*>(base + ws.split_o);
+  plan.split_lse = reinterpret_cast<float*>(base + ws.split_lse);
   return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, fresh_row,
                        need_ctx + kCtxPadRows, plan.kctx, plan.vctx, plan.ctx_rows, stream);
 }

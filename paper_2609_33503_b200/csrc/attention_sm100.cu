@@ -14,6 +14,7 @@
 // flag, records RELAXKV_ERR_TIMEOUT in the device status word and the block tears down normally.
 #include "attention_common.cuh"
 #include "sm100_ptx.cuh"
+#include <algorithm>
 
 namespace relaxkv {
 
@@ -50,7 +51,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        const int* __restrict__ u_pos, const int* __restrict__ u_cu,
                        const int* __restrict__ r_rank, const int* __restrict__ r_cu,
                        long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
-                       DeviceStatus* st) {
+                       float* __restrict__ part_o, float* __restrict__ part_lse, DeviceStatus* st) {
   using L = AttnSmem<D>;
   constexpr int kHalves = L::kHalves;
   constexpr uint32_t kTmemCols = 512;          // S_A | S_B | O_A | O_B, 128 columns each (O uses D of them)
@@ -97,6 +98,25 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
   }
   const int n_kv_max = max(n_kv[0], n_kv[1]);
+  // Context split (gridDim.y > 1, used when there are too few query tiles to fill the GPU): this block walks the
+  // context tiles [j0, j0 + chunk) of its pair and leaves a normalised partial result + its log-sum-exp.
+  const int n_splits = (int)gridDim.y, split = (int)blockIdx.y;
+  const int chunk = (n_kv_max + n_splits - 1) / n_splits;
+  const int j0 = split * chunk;
+  int n_my[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) n_my[x] = max(0, min(n_kv[x], j0 + chunk) - j0);
+  const int n_my_max = max(n_my[0], n_my[1]);
+  if (n_my_max == 0) {                        // nothing of this pair's context falls into this split
+    if (n_splits > 1 && threadIdx.x < 2 * kBM) {
+      const int x = threadIdx.x >> 7, row = threadIdx.x & 127, t_local = row / G;
+      if (row < tile_targets * G && t_local < n_valid[x]) {
+        const long long orow = q_row_base + x * tile_targets + t_local;
+        part_lse[((long long)split * n_target_rows + orow) * H + hd * G + (row - t_local * G)] = -INFINITY;
+      }
+    }
+    return;
+  }
 
   // ---- shared memory -----------------------------------------------------------------------------
   extern __shared__ uint8_t smem_raw[];
@@ -156,10 +176,10 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int hf = 0; hf < kHalves; ++hf)
           tma_load_3d(q_smem + (x * kHalves + hf) * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G,
                       (int)(q_row_base + x * tile_targets));
-      for (int u = 0; u < 2 * n_kv_max; ++u) {                // u = 2*j + (0: K, 1: V)
+      for (int u = 0; u < 2 * n_my_max; ++u) {                // u = 2*j + (0: K, 1: V), j counted from j0
         const int s = u % kRing;
         if (u >= kRing && !mbar_wait(bar_empty + 8 * s, ((u / kRing) - 1) & 1, abort_flag)) break;
-        const int row = (int)(ctx_base + (long long)(u >> 1) * kBN);
+        const int row = (int)(ctx_base + (long long)(j0 + (u >> 1)) * kBN);
         const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
         mbar_expect_tx(bar_full + 8 * s, L::kTileBytes);
         for (int hf = 0; hf < kHalves; ++hf)
@@ -196,24 +216,24 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (!mbar_wait(bar_pfull_hi + 8 * x, j & 1, abort_flag)) return false;
         tc_fence_after();
         mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128 + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
-        if (j == n_kv[x] - 1) mma_commit(bar_ofinal + 8 * x);
+        if (j == n_my[x] - 1) mma_commit(bar_ofinal + 8 * x);
         return true;
       };
-      if (ok && n_kv[0] > 0) ok = issue_qk(0, 0, true);
-      if (ok && n_kv[1] > 0) ok = issue_qk(1, 0, n_kv[0] == 0);
+      if (ok && n_my[0] > 0) ok = issue_qk(0, 0, true);
+      if (ok && n_my[1] > 0) ok = issue_qk(1, 0, n_my[0] == 0);
       if (ok) mma_commit(bar_empty + 8 * 0);                   // K_0's buffer: free once both S tiles are done
-      for (int j = 0; ok && j < n_kv_max; ++j) {
-        const bool a_pv = j < n_kv[0], a_qk = j + 1 < n_kv[0];
+      for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0
+        const bool a_pv = j < n_my[0], a_qk = j + 1 < n_my[0];
         if (a_pv) {
           if (!(ok = issue_pv(0, j, true))) break;
           if (a_qk && !(ok = issue_qk(0, j + 1, true))) break;
         }
-        if (j < n_kv[1]) {
+        if (j < n_my[1]) {
           if (!(ok = issue_pv(1, j, !a_pv))) break;
         }
         mma_commit(bar_empty + 8 * ((2 * j + 1) % kRing));     // V_j
-        if (j + 1 < n_kv[1] && !(ok = issue_qk(1, j + 1, !a_qk))) break;
-        if (j + 1 < n_kv_max) mma_commit(bar_empty + 8 * ((2 * j + 2) % kRing));   // K_{j+1}
+        if (j + 1 < n_my[1] && !(ok = issue_qk(1, j + 1, !a_qk))) break;
+        if (j + 1 < n_my_max) mma_commit(bar_empty + 8 * ((2 * j + 2) % kRing));   // K_{j+1}
       }
     }
   }
@@ -241,7 +261,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t t_s = lane_base + x * 128, t_o = lane_base + 256 + x * 128;
     const uint32_t my_sfull = bar_sfull + 8 * x, my_pfull = bar_pfull + 8 * x;
-    const int my_n = n_kv[x];
+    const int my_n = n_my[x];
     float m = -INFINITY, z = 0.f;
     bool ok = true;
     for (int j = 0; j < my_n; ++j) {
@@ -253,7 +273,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
       for (int c = 0; c < kBN / 32; ++c) tmem_ld32(t_s + c * 32, &s[c * 32]);
       tmem_wait_ld();
-      const int col0 = j * kBN;
+      const int col0 = (j0 + j) * kBN;
       if (col0 + kBN - 1 > limit) {
 #pragma unroll
         for (int i = 0; i < kBN; ++i)
@@ -274,7 +294,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                              fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
       const float m_new = mx * scale_log2;
       if (j == 0) {
-        m = m_new;
+        m = fmaxf(m_new, -1.0e30f);           // a row whose first tile of this split is fully masked keeps a finite reference
       } else {
         // S_x(j) is complete, hence so is O_x += P_x V_{j-1}: O_x may be rescaled here
         const bool need = m_new > m + kRescaleThreshold;
@@ -334,30 +354,55 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     if (ok && my_n > 0) {
       tc_fence_after();
-      const float inv = row_empty ? 0.f : 1.f / z;              // an empty context is defined as a zero output row
+      const bool none = row_empty || !(z > 0.f);                // an empty context is defined as a zero output row
+      const float inv = none ? 0.f : 1.f / z;
+      const float lse = none ? -INFINITY : (m + log2f(z)) * kLn2A;
       const long long orow = q_row_base + x * tile_targets + t_local;
-      uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
+      if (n_splits == 1) {
+        uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(t_o + c * 32, o);
-        tmem_wait_ld();
-        if (row_valid) {
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(t_o + c * 32, o);
+          tmem_wait_ld();
+          if (row_valid) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint32_t w[4];
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv,
-                                                        __uint_as_float(o[i + 2 * e + 1]) * inv);
-              w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv,
+                                                          __uint_as_float(o[i + 2 * e + 1]) * inv);
+                w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(optr + c * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            *reinterpret_cast<uint4*>(optr + c * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
+        if (row_valid && lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = lse;
+      } else {
+        // partial result of this split: fp32, normalised by this split's own sum
+        const long long slot = ((long long)split * n_target_rows + orow) * H + hd * G + j_head;
+        float* optr = part_o + slot * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(t_o + c * 32, o);
+          tmem_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(optr + c * 32 + i) =
+                  make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv, __uint_as_float(o[i + 2]) * inv,
+                              __uint_as_float(o[i + 3]) * inv);
+          }
+        }
+        if (row_valid) part_lse[slot] = lse;
       }
-      if (row_valid && lse_out)
-        lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = row_empty ? -INFINITY : (m + log2f(z)) * kLn2A;
+    } else if (ok && my_n == 0 && n_splits > 1 && row_valid) {
+      // this tile's context ends before the split begins (the pair's other tile still has work here)
+      const long long orow = q_row_base + x * tile_targets + t_local;
+      part_lse[((long long)split * n_target_rows + orow) * H + hd * G + j_head] = -INFINITY;
     }
   }
 
@@ -429,6 +474,44 @@ __global__ void wait_timeout_probe_kernel(DeviceStatus* st) {
   }
 }
 
+// Merges the partial results of a context split: out = sum_s w_s O_s / sum_s w_s with w_s = exp(lse_s - max lse).
+// One warp per (target row, query head); rows past the true target count are left alone.
+__global__ void combine_splits_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits,
+                                      long long n_target_rows, int H, int D, const int* __restrict__ r_cu, int n_req,
+                                      uint16_t* __restrict__ out, float* __restrict__ lse_out) {
+  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const long long rows_true = r_cu[n_req] - r_cu[0];
+  if (w >= rows_true * H) return;
+  const long long row = w / H;
+  const int h = (int)(w - row * H);
+  float mx = -INFINITY;
+  for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_lse[((long long)sp * n_target_rows + row) * H + h]);
+  const int per = D / 32;                       // 2 or 4 consecutive floats per lane
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float den = 0.f;
+  if (mx > -INFINITY) {
+    for (int sp = 0; sp < n_splits; ++sp) {     // fixed order: reproducible
+      const long long slot = ((long long)sp * n_target_rows + row) * H + h;
+      const float l = part_lse[slot];
+      if (l == -INFINITY) continue;
+      const float wgt = __expf(l - mx);
+      den += wgt;
+      const float* o = part_o + slot * D + lane * per;
+      for (int e = 0; e < per; ++e) acc[e] += wgt * o[e];
+    }
+  }
+  const float inv = den > 0.f ? 1.f / den : 0.f;
+  uint16_t* optr = out + (row * H + h) * D + lane * per;
+  for (int e = 0; e < per; e += 2) {
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
+    *reinterpret_cast<uint32_t*>(optr + e) = *reinterpret_cast<uint32_t*>(&h2);
+  }
+  if (lane == 0 && lse_out) lse_out[(long long)h * n_target_rows + row] = den > 0.f ? mx + logf(den) : -INFINITY;
+}
+
+static int g_forced_splits = 0;      // 0: chosen from the launch size; > 0: forced (test hook)
+
 // ---- host side ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -485,6 +568,24 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   long long ctx_rows_used = 0;
   for (int b = 0; b < B; ++b) ctx_rows_used += plan.rt.bound_b[b];
   const int head_inner = (ctx_rows_used * (long long)row_kv * 2 <= (40ll << 20)) ? 1 : 0;
+  // Too few query tiles to fill the GPU (a query prefill, a decode step, a deep layer with few targets): split
+  // every pair's context over several blocks and merge the partial results afterwards.
+  static int sm_count[64] = {0};
+  int dev0 = 0;
+  if (cudaGetDevice(&dev0) != cudaSuccess || dev0 < 0 || dev0 >= 64) return RELAXKV_ERR_CUDA;
+  if (sm_count[dev0] == 0 && cudaDeviceGetAttribute(&sm_count[dev0], cudaDevAttrMultiProcessorCount, dev0) != cudaSuccess)
+    return RELAXKV_ERR_CUDA;
+  long long max_tiles = 1;
+  for (int b = 0; b < B; ++b) max_tiles = std::max<long long>(max_tiles, (plan.rt.bound_b[b] + kBN - 1) / kBN);
+  long long n_splits = 1;
+  if (g_forced_splits > 0) {
+    n_splits = g_forced_splits;
+  } else if (grid < sm_count[dev0]) {
+    n_splits = std::min<long long>((2ll * sm_count[dev0] + grid - 1) / grid, std::max<long long>(1, max_tiles / 4));
+  }
+  n_splits = std::min<long long>(n_splits, kMaxCtxSplits);
+  n_splits = std::min<long long>(n_splits, kSplitRowsCap / n_target_rows);   // partial slots: [split][row of the call]
+  if (n_splits < 1) n_splits = 1;
   auto kern = attention_sm100_kernel<D>;
   static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
   int dev = 0;
@@ -494,9 +595,14 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
       return RELAXKV_ERR_CUDA;
     attr_done[dev] = true;
   }
-  kern<<<(unsigned)grid, kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
+  kern<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
       tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
-      r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, st);
+      r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
+  relaxkv_status rc = launch_ok();
+  if (rc != RELAXKV_OK || n_splits == 1) return rc;
+  const long long warps = plan.sum_targets * H;
+  combine_splits_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(
+      plan.split_o, plan.split_lse, (int)n_splits, n_target_rows, H, D, r_cu_layer, B, static_cast<uint16_t*>(out), lse_out);
   return launch_ok();
 }
 
@@ -519,6 +625,12 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention(
   if (shape->head_dim == 128)
     return launch_attention<128>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
   return launch_attention<64>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
+}
+
+extern "C" relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits) {
+  if (n_splits < 0 || n_splits > kMaxCtxSplits) return RELAXKV_ERR_INVALID_ARG;
+  g_forced_splits = n_splits;
+  return RELAXKV_OK;
 }
 
 extern "C" relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream) {

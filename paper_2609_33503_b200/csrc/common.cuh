@@ -108,6 +108,8 @@ constexpr int kScoreSplitsMax = 64;   // key-range splits of the scoring passes 
 constexpr int kScoreMaxRows = 640;    // query rows (token x head-in-group) resident per scoring CTA
 constexpr int kScoreTokBox = 8;       // query tokens per TMA box of the scoring kernel
 constexpr int kCtxPadRows = 128;      // zero rows after the materialised context
+constexpr int kSplitRowsCap = 2048;   // (target rows) x (context splits) the split workspace holds
+constexpr int kMaxCtxSplits = 32;
 
 constexpr int kScoreLayersPerLaunch = 48;   // layers scored by one launch (their tensor maps travel as parameters)
 
@@ -140,6 +142,8 @@ struct WsLayout {
   size_t kctx, vctx; long long ctx_rows_cap;
   // explicit-list attention: limit [sumT] i32 | fresh_row [sumT] i32
   size_t list_limit, list_fresh;
+  // context split across blocks (few targets): partial O [kSplitRowsCap, H, D] f32 | partial lse [kSplitRowsCap, H] f32
+  size_t split_o, split_lse;
   // scoring (per launch of Lc <= kScoreLayersPerLaunch layers): lse [Lc, H, sumQ] f32 |
   // part [Lc, 2*n_splits, H, sumQ] float2 | colpart [Lc, 2*H_kv*max_blocks, sumT] f32
   size_t lse, part, colpart;
@@ -159,6 +163,8 @@ inline WsLayout ws_layout(const relaxkv_shape* s, int n_layers) {
   w.vctx = a; a = align_up(a + (size_t)w.ctx_rows_cap * row_bytes, 1024);
   w.list_limit = a; a = align_up(a + (size_t)sum_t * 4, 256);
   w.list_fresh = a; a = align_up(a + (size_t)sum_t * 4, 256);
+  w.split_o = a; a = align_up(a + (size_t)kSplitRowsCap * s->n_q_heads * s->head_dim * 4, 256);
+  w.split_lse = a; a = align_up(a + (size_t)kSplitRowsCap * s->n_q_heads * 4, 256);
   size_t attn_total = a;
   a = 0;
   const int lc_max = n_layers < kScoreLayersPerLaunch ? n_layers : kScoreLayersPerLaunch;

@@ -241,6 +241,34 @@ def test_attention_matches_oracle(case, simt, full_prefix):
         check_attention(case, l, out, lse, full_prefix)
 
 
+@pytest.mark.parametrize("n_splits", [1, 2, 5, 32])
+def test_context_split_matches_oracle(case, n_splits):
+    """Few query tiles: the context of every tile pair is split over several blocks and the partial results are
+    merged by their log-sum-exp.  Forced here to 1 (never), 2, 5 and 32 splits (more splits than some pairs have
+    context tiles: empty splits), in both context modes, against the oracle; the rows past the true target count
+    of a loosely bounded call stay untouched."""
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    B().relaxkv_debug_set_attention_splits(n_splits)
+    try:
+        for l in range(case.w.n_layers):
+            for full_prefix in (False, True):
+                out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
+                check_attention(case, l, out, lse, full_prefix)
+        f = case.fresh[0]
+        n = f.q_new.shape[0]
+        pad = 7
+        q_pad = torch.cat([f.q_new, torch.zeros(pad, *f.q_new.shape[1:], dtype=f.q_new.dtype, device=f.q_new.device)])
+        out = torch.full_like(q_pad, 3.0)
+        s.attention(0, case.cache_views()[0], q_pad, f.k_new, f.v_new, out, list(case.w.ctx_lens), list(case.w.ctx_lens))
+        assert_status_ok()
+        assert torch.all(out[n:] == 3.0)
+        exact, _ = run_attention(case, s, 0, B().CTX_UNION, simt=False)
+        assert torch.equal(out[:n], exact)
+    finally:
+        B().relaxkv_debug_set_attention_splits(0)
+
+
 def test_attention_orders_agree_and_is_deterministic(case):
     """Update-then-attend from the cache equals mix-then-attend (Algorithm 1's order), bit for bit;
     two runs give identical bits."""
@@ -300,17 +328,28 @@ def test_edge_sizes(ctx, q, ratio):
 
 
 def test_loose_host_bounds_give_the_same_result(case):
-    """Host bounds may be loose (|R_l| <= |U| <= T_c): same bits as with exact bounds."""
+    """Host bounds may be loose (|R_l| <= |U| <= T_c).  With the same context split the bits are those of the
+    exact bounds; when the launch size picks another split count only the summation order changes."""
     w = case.w
     s = case.make_session()
     s.build_active_sets(case.anchors_tensor())
     l = 0
     f = case.fresh[l]
-    exact, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
-    out = torch.zeros_like(f.q_new)
-    s.attention(l, case.cache_views()[l], f.q_new, f.k_new, f.v_new, out, list(w.ctx_lens), list(w.ctx_lens))
-    assert_status_ok()
-    assert torch.equal(out, exact)
+    for forced in (1, 0):
+        B().relaxkv_debug_set_attention_splits(forced)
+        try:
+            exact, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
+            out = torch.zeros_like(f.q_new)
+            lse = torch.zeros(w.n_q_heads, f.q_new.shape[0], dtype=torch.float32, device=case.device)
+            s.attention(l, case.cache_views()[l], f.q_new, f.k_new, f.v_new, out, list(w.ctx_lens), list(w.ctx_lens), lse_out=lse)
+            assert_status_ok()
+        finally:
+            B().relaxkv_debug_set_attention_splits(0)
+        if forced == 1:
+            assert torch.equal(out, exact)
+        else:
+            check_attention(case, l, out, lse, False)
+            assert float((out.float() - exact.float()).abs().max()) <= 2e-2
 
 
 def test_bad_index_lists_are_reported_not_faulted():
