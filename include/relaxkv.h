@@ -334,6 +334,25 @@ relaxkv_status relaxkv_sparse_ctx_attention_simt(
     void* workspace, size_t workspace_bytes, relaxkv_stream stream);
 
 /*
+ * Attention of given token positions over the cache's own causal prefix, cache only: target t of request b,
+ * at position p = tgt_pos[tgt_cu[b] + t], attends to every cache entry j <= p of its request.  This is the pass
+ * the paper runs after the repair loop (the user query's prefill rows and the first decode step read the
+ * repaired cache; Section 3.4 and the TTFT protocol of the reproducibility appendix): the caller has appended
+ * the K/V of those tokens to the cache, `shape->h_ctx_len[b]` counts them.  No context is gathered: the
+ * kernel's tiled loads read the cache through its strides, so the call moves K and V once.
+ *   q_new  device bf16 [n_target_rows, H, D], rows in tgt order, requests packed
+ *   tgt_pos / tgt_cu  device int32: ascending positions per request, packed; offsets [B + 1], tgt_cu[0] = 0
+ *   h_max_targets  host [B] upper bounds on the target counts
+ *   out  device bf16 [n_target_rows, H, D]; lse_out optional device fp32 [H, n_target_rows]
+ * The cache must hold max_b(h_req_token_offset[b] + h_ctx_len[b]) token rows.  Errors as for
+ * relaxkv_sparse_ctx_attention (positions out of range are reported in the device status word).
+ */
+relaxkv_status relaxkv_cache_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q_new,
+    const int32_t* tgt_pos, const int32_t* tgt_cu, int64_t n_target_rows, const int32_t* h_max_targets,
+    void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/*
  * Test utility (the paper has no counterpart).  The attention calls split every query tile's context over
  * several thread blocks when there are too few query tiles to fill the GPU (a query prefill, a decode step, a
  * layer with few active targets) and merge the partial results by their log-sum-exp; the split count is

@@ -24,7 +24,7 @@ ENTRY_POINTS = (
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_debug_set_attention_splits",
-    "relaxkv_list_attention",
+    "relaxkv_list_attention", "relaxkv_cache_attention",
     "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
@@ -252,6 +252,16 @@ def relaxkv_list_attention(shape: Shape, cache: CacheView, q_new: torch.Tensor, 
                                         _i32(max_targets), _i32(max_ctx), _ptr(out), _ptr(lse_out), _ptr(workspace),
                                         ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)),
            "relaxkv_list_attention")
+
+
+def relaxkv_cache_attention(shape: Shape, cache: CacheView, q_new: torch.Tensor, tgt_pos: torch.Tensor, tgt_cu: torch.Tensor,
+                            max_targets: Sequence[int], out: torch.Tensor, workspace: torch.Tensor,
+                            lse_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(lib().relaxkv_cache_attention(shape.ref(), cache.ref(), _ptr(q_new), _ptr(tgt_pos), _ptr(tgt_cu),
+                                         ctypes.c_int64(q_new.shape[0]), _i32(max_targets), _ptr(out), _ptr(lse_out),
+                                         _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                         _stream(stream)),
+           "relaxkv_cache_attention")
 
 
 def relaxkv_scatter_kv_lists(shape: Shape, cache: CacheView, k_new: torch.Tensor, v_new: torch.Tensor,

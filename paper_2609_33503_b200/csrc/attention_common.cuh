@@ -13,6 +13,10 @@ struct AttnPlan {
   long long sum_targets;  // sum of the host bounds on |R_{l,b}|
   float* split_o;         // workspace for a context split across blocks: [kSplitRowsCap, H, D] and [kSplitRowsCap, H]
   float* split_lse;
+  // what the attention kernel's K/V tensor maps cover: the materialised context, or the cache itself
+  const void* k_base; const void* v_base;
+  unsigned long long kv_token_stride_bytes, kv_head_stride_bytes;
+  int dense_ctx;          // 1: context = the cache's own rows (request b starts at rt.tok_off[b]), limits are positions
 };
 
 // Validates the arguments of an attention call and enqueues the gather of the mixed context into
@@ -57,6 +61,11 @@ inline relaxkv_status prepare_attention(
   plan.ctx_rows = ws.ctx_rows_cap;
   plan.split_o = reinterpret_cast<float*>(base + ws.split_o);
   plan.split_lse = reinterpret_cast<float*>(base + ws.split_lse);
+  plan.k_base = plan.kctx;
+  plan.v_base = plan.vctx;
+  plan.kv_head_stride_bytes = (unsigned long long)shape->head_dim * 2;
+  plan.kv_token_stride_bytes = (unsigned long long)shape->n_kv_heads * shape->head_dim * 2;
+  plan.dense_ctx = 0;
   return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, fresh_row,
                        need_ctx + kCtxPadRows, plan.kctx, plan.vctx, plan.ctx_rows, stream);
 }

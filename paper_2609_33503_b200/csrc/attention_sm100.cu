@@ -47,7 +47,7 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
-                       int mode, int allow_empty, int head_inner, int H, int Hkv, int tile_targets, float scale_log2,
+                       int mode, int allow_empty, int head_inner, int dense_ctx, int H, int Hkv, int tile_targets, float scale_log2,
                        const int* __restrict__ u_pos, const int* __restrict__ u_cu,
                        const int* __restrict__ r_rank, const int* __restrict__ r_cu,
                        long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
@@ -69,7 +69,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int b = find_segment(rt.tile_cu, B, tt);
   const int p_rev = tt - rt.tile_cu[b];
   const int nr = r_cu[b + 1] - r_cu[b];
-  const int nu = u_cu[b + 1] - u_cu[b];
+  // dense_ctx: the context is the cache itself (every position of the request), a target's limit is its position
+  const int nu = dense_ctx ? rt.ctx_len[b] : (u_cu[b + 1] - u_cu[b]);
   const int pair_targets = 2 * tile_targets;
   const int n_pairs_true = (nr + pair_targets - 1) / pair_targets;
   if (p_rev >= n_pairs_true) return;
@@ -81,7 +82,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int pair = n_pairs_true - 1 - p_rev;
   const int rho0 = pair * pair_targets;                       // first target of tile A
   const int ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
-  const long long ctx_base = (mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b];
+  const long long ctx_base = dense_ctx ? rt.tok_off[b] : ((mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b]);
   const long long q_row_base = (long long)(r_cu[b] - r_cu[0]) + rho0;
   // valid targets and context tiles of each query tile
   int n_valid[2], n_kv[2];
@@ -559,8 +560,10 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   CUtensorMap tm_q, tm_k, tm_v;
   const uint64_t row_q = (uint64_t)H * D * 2, row_kv = (uint64_t)Hkv * D * 2;
   if (!make_map_3d(&tm_q, q_new, D, H, (uint64_t)n_target_rows, (uint64_t)D * 2, row_q, (uint32_t)G, (uint32_t)tile_targets) ||
-      !make_map_3d(&tm_k, plan.kctx, D, Hkv, (uint64_t)plan.ctx_rows, (uint64_t)D * 2, row_kv, 1u, (uint32_t)kBN) ||
-      !make_map_3d(&tm_v, plan.vctx, D, Hkv, (uint64_t)plan.ctx_rows, (uint64_t)D * 2, row_kv, 1u, (uint32_t)kBN))
+      !make_map_3d(&tm_k, plan.k_base, D, Hkv, (uint64_t)plan.ctx_rows, plan.kv_head_stride_bytes, plan.kv_token_stride_bytes, 1u,
+                   (uint32_t)kBN) ||
+      !make_map_3d(&tm_v, plan.v_base, D, Hkv, (uint64_t)plan.ctx_rows, plan.kv_head_stride_bytes, plan.kv_token_stride_bytes, 1u,
+                   (uint32_t)kBN))
     return RELAXKV_ERR_CUDA;
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
@@ -581,7 +584,8 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   if (g_forced_splits > 0) {
     n_splits = g_forced_splits;
   } else if (grid < sm_count[dev0]) {
-    n_splits = std::min<long long>((2ll * sm_count[dev0] + grid - 1) / grid, std::max<long long>(1, max_tiles / 4));
+    // one full wave: as many splits as whole blocks fit the SMs, each at least four context tiles long
+    n_splits = std::min<long long>(std::max<long long>(1, sm_count[dev0] / grid), std::max<long long>(1, max_tiles / 4));
   }
   n_splits = std::min<long long>(n_splits, kMaxCtxSplits);
   n_splits = std::min<long long>(n_splits, kSplitRowsCap / n_target_rows);   // partial slots: [split][row of the call]
@@ -596,7 +600,7 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
     attr_done[dev] = true;
   }
   kern<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
-      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
+      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA, u_pos, u_cu, r_rank,
       r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
   relaxkv_status rc = launch_ok();
   if (rc != RELAXKV_OK || n_splits == 1) return rc;
@@ -689,4 +693,48 @@ extern "C" relaxkv_status relaxkv_list_attention(
                                  lse_out, stream, 1);
   return launch_attention<64>(shape, RELAXKV_CTX_UNION, plan, q_new, ctx_pos, ctx_cu, limit, tgt_cu, n_target_rows, out,
                               lse_out, stream, 1);
+}
+
+// Attention of given token positions over the cache's own causal prefix (cache only, no gather): the tensor maps
+// cover the cache, a target's causal limit is its position.
+extern "C" relaxkv_status relaxkv_cache_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q_new,
+    const int32_t* tgt_pos, const int32_t* tgt_cu, int64_t n_target_rows, const int32_t* h_max_targets,
+    void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if ((rc = check_cache(shape, cache, true)) != RELAXKV_OK) return rc;
+  if (!q_new || !out || !tgt_pos || !tgt_cu || !h_max_targets || !workspace) return RELAXKV_ERR_INVALID_ARG;
+  if (!aligned16(q_new) || !aligned16(out) || n_target_rows < 1) return RELAXKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return RELAXKV_ERR_INVALID_ARG;
+  const WsLayout ws = ws_layout(shape, 1);
+  if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
+  AttnPlan plan;
+  fill_req_table(plan.rt, shape, cache, nullptr);
+  plan.sum_targets = 0;
+  long long cache_rows = 0;
+  for (int b = 0; b < shape->n_req; ++b) {
+    if (h_max_targets[b] < 0 || h_max_targets[b] > shape->h_ctx_len[b]) return RELAXKV_ERR_INVALID_ARG;
+    plan.rt.bound_a[b] = h_max_targets[b];
+    plan.rt.bound_b[b] = shape->h_ctx_len[b];
+    plan.sum_targets += h_max_targets[b];
+    cache_rows = std::max<long long>(cache_rows, (long long)cache->h_req_token_offset[b] + shape->h_ctx_len[b]);
+  }
+  if (plan.sum_targets > 0x7fffffffLL || cache_rows > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  char* base = static_cast<char*>(workspace);
+  plan.kctx = nullptr; plan.vctx = nullptr;
+  plan.split_o = reinterpret_cast<float*>(base + ws.split_o);
+  plan.split_lse = reinterpret_cast<float*>(base + ws.split_lse);
+  plan.k_base = cache->k; plan.v_base = cache->v;
+  plan.kv_head_stride_bytes = (unsigned long long)cache->head_stride * 2;
+  plan.kv_token_stride_bytes = (unsigned long long)cache->token_stride * 2;
+  plan.ctx_rows = cache_rows;
+  plan.dense_ctx = 1;
+  // lists: targets by position (their "rank" in the dense context), counts from tgt_cu; u_pos / u_cu are not read
+  if (shape->head_dim == 128)
+    return launch_attention<128>(shape, RELAXKV_CTX_UNION, plan, q_new, nullptr, nullptr, tgt_pos, tgt_cu, n_target_rows, out,
+                                 lse_out, stream);
+  return launch_attention<64>(shape, RELAXKV_CTX_UNION, plan, q_new, nullptr, nullptr, tgt_pos, tgt_cu, n_target_rows, out,
+                              lse_out, stream);
 }

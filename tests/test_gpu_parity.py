@@ -551,6 +551,57 @@ def test_query_prefill_lse_replaces_the_statistics_pass():
     check_anchor_band(ref_raw, case.k[0], s.anchors.cpu().numpy()[0])
 
 
+@pytest.mark.parametrize("head_major", [False, True])
+@pytest.mark.parametrize("n_splits", [0, 1, 3])
+def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
+    """The pass after the repair loop: query rows (and a single decode token) attend to the cache's own causal
+    prefix, read through the cache's strides without a gather.  Three requests in one call, token-major and
+    head-major caches with a gap between the requests' rows, against the oracle's explicit-list attention with
+    every position as context."""
+    H, Hkv, D = 16, 4, 128
+    lens, n_tgt = (1500, 300, 2200), (37, 1, 64)                 # the middle request is a decode step: one row
+    offs = [0, 1600, 2000]                                        # rows 1500..1599 and 1900..1999 belong to nobody
+    rows = 4300
+    g = torch.Generator(device="cpu").manual_seed(5)
+    k_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    v_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    if head_major:
+        k_all = k_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
+        v_all = v_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
+    q = torch.randn(sum(n_tgt), H, D, generator=g).to(torch.bfloat16).cuda()
+    # targets: the last tokens of each request (the query suffix), ascending
+    tgt = [np.arange(t - n, t, dtype=np.int32) for t, n in zip(lens, n_tgt)]
+    tgt_pos = torch.from_numpy(np.concatenate(tgt)).cuda()
+    tgt_cu = torch.tensor(np.concatenate([[0], np.cumsum(n_tgt)]).astype(np.int32)).cuda()
+    shape = B().Shape(H, Hkv, D, list(lens), None, D ** -0.5)
+    ws = torch.empty(B().relaxkv_workspace_bytes(shape, 1) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.zeros_like(q)
+    lse = torch.zeros(H, q.shape[0], dtype=torch.float32, device="cuda")
+    B().relaxkv_debug_set_attention_splits(n_splits)
+    try:
+        B().relaxkv_cache_attention(shape, B().CacheView(k_all, v_all, offs), q, tgt_pos, tgt_cu, list(n_tgt), out, ws, lse_out=lse)
+        assert_status_ok()
+    finally:
+        B().relaxkv_debug_set_attention_splits(0)
+    lo = 0
+    for b in range(3):
+        kb = inputs.bf16_bits(k_all[offs[b]:offs[b] + lens[b]].contiguous())
+        vb = inputs.bf16_bits(v_all[offs[b]:offs[b] + lens[b]].contiguous())
+        qb = inputs.bf16_bits(q[lo:lo + n_tgt[b]])
+        ref, ref_lse = orc.list_attention(kb, vb, qb, None, None, np.arange(lens[b]), tgt[b], D ** -0.5)
+        mx, mean = attention_errors(out[lo:lo + n_tgt[b]], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (b, mx, mean)
+        np.testing.assert_allclose(lse[:, lo:lo + n_tgt[b]].cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+        lo += n_tgt[b]
+    # a position past the request's end is reported, not read
+    bad = tgt_pos.clone()
+    bad[0] = lens[0]
+    B().relaxkv_cache_attention(shape, B().CacheView(k_all, v_all, offs), q, bad, tgt_cu, list(n_tgt), out, ws)
+    st, _ = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX
+
+
 def test_head_sharded_selection_on_one_gpu():
     """The head-sharded selection path, its ranks run one after the other on this GPU (their kernels never wait
     on one another): partial scores of the two KV-head shards average to the unsharded scores, and the anchors
