@@ -1,10 +1,13 @@
 // y = x W^T (+ residual) on the Blackwell tensor cores: the projections of the active targets' block work
 // (Algorithm 1, steps 16 and 20).  x [M, K], W [N, K] (the [out, in] layout), y [M, N], bf16 with fp32
-// accumulation in TMEM.  CTA tile 128 x 256, K blocks of 64 through a 4-stage TMA ring (128-byte swizzle),
-// one MMA issuer thread (tcgen05.mma M=128, N=256, K=16), four epilogue warps (thread = row = TMEM lane).
-// Tiles are walked in groups of 16 row tiles so that a wave's working set (x rows + W rows) stays in L2.
+// accumulation in TMEM.  Persistent kernel, one CTA per SM: CTA tile 128 x 256, K blocks of 64 through a
+// 4-stage TMA ring (128-byte swizzle) that runs on across tiles, one MMA issuer thread (tcgen05.mma M=128,
+// N=256, K=16), two 256-column accumulators in TMEM so that the four epilogue warps (thread = row = TMEM
+// lane) drain tile i while the tensor pipe works on tile i+1.  Tiles are walked in groups of 16 row tiles so
+// that a wave's working set (x rows + W rows) stays in L2.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include <algorithm>
 
 namespace relaxkv {
 
@@ -16,38 +19,44 @@ bool make_map_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uin
 constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64, kGemmStages = 4, kGemmThreads = 192, kGemmGroupM = 16;
 constexpr int kGemmABytes = kGemmBM * kGemmBK * 2, kGemmBBytes = kGemmBN * kGemmBK * 2;
 constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;
-constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 8 * (2 * kGemmStages + 1) + 16 + 1024;
+constexpr int kGemmBars = 2 * kGemmStages + 4;           // full, empty per stage; accumulator full, empty x 2
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 8 * kGemmBars + 16 + 1024;
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   long long M, int N, int K, uint16_t* __restrict__ y, const uint16_t* __restrict__ residual,
                   DeviceStatus* st) {
-  // ---- which tile (grouped order: kGemmGroupM row tiles x all column tiles at a time) ----
   const int tiles_m = (int)((M + kGemmBM - 1) / kGemmBM), tiles_n = (N + kGemmBN - 1) / kGemmBN;
-  const int pid = blockIdx.x;
-  const int per_group = kGemmGroupM * tiles_n;
-  const int group = pid / per_group, first_m = group * kGemmGroupM;
-  const int group_m = min(tiles_m - first_m, kGemmGroupM);
-  const int tm = first_m + (pid % per_group) % group_m, tn = (pid % per_group) / group_m;
+  const long long n_tiles = (long long)tiles_m * tiles_n;
   if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;
+  // tile t of the grouped order: kGemmGroupM row tiles x all column tiles at a time
+  auto tile_of = [&](long long t, int& tm, int& tn) {
+    const int per_group = kGemmGroupM * tiles_n;
+    const int group = (int)(t / per_group), first_m = group * kGemmGroupM;
+    const int group_m = min(tiles_m - first_m, kGemmGroupM);
+    const int r = (int)(t - (long long)group * per_group);
+    tm = first_m + r % group_m;
+    tn = r / group_m;
+  };
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bar0 = base + kGemmStages * kGemmStageBytes;
-  const uint32_t bar_full = bar0, bar_empty = bar0 + 8 * kGemmStages, bar_acc = bar0 + 16 * kGemmStages;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kGemmStages * kGemmStageBytes + 8 * (2 * kGemmStages + 1));
+  const uint32_t bar_full = bar0, bar_empty = bar0 + 8 * kGemmStages;
+  const uint32_t bar_acc_full = bar0 + 16 * kGemmStages, bar_acc_empty = bar_acc_full + 16;     // [2] each
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kGemmStages * kGemmStageBytes + 8 * kGemmBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(const_cast<uint32_t*>(tmem_slot) + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kGemmStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-    mbar_init(bar_acc, 1);
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 128); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
   }
-  if (warp == 5) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256); tmem_relinquish(); }
+  if (warp == 5) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -55,38 +64,60 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int n_k = (K + kGemmBK - 1) / kGemmBK;
 
   if (warp == 4) {
+    // ---- TMA producer: the ring index runs on from tile to tile ----
     if (lane == 0) {
       prefetch_tensormap(&tm_a); prefetch_tensormap(&tm_b);
-      for (int kt = 0; kt < n_k; ++kt) {
-        const int s = kt % kGemmStages;
-        if (kt >= kGemmStages && !mbar_wait(bar_empty + 8 * s, ((kt / kGemmStages) - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(bar_full + 8 * s, kGemmStageBytes);
-        tma_load_3d(base + s * kGemmStageBytes, &tm_a, bar_full + 8 * s, kt * kGemmBK, tm * kGemmBM, 0);
-        tma_load_3d(base + s * kGemmStageBytes + kGemmABytes, &tm_b, bar_full + 8 * s, kt * kGemmBK, tn * kGemmBN, 0);
+      long long it = 0;
+      for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        int tm, tn;
+        tile_of(t, tm, tn);
+        bool ok = true;
+        for (int kt = 0; kt < n_k; ++kt, ++it) {
+          const int s = (int)(it % kGemmStages);
+          if (it >= kGemmStages && !(ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kGemmStages) - 1) & 1, abort_flag))) break;
+          mbar_expect_tx(bar_full + 8 * s, kGemmStageBytes);
+          tma_load_3d(base + s * kGemmStageBytes, &tm_a, bar_full + 8 * s, kt * kGemmBK, tm * kGemmBM, 0);
+          tma_load_3d(base + s * kGemmStageBytes + kGemmABytes, &tm_b, bar_full + 8 * s, kt * kGemmBK, tn * kGemmBN, 0);
+        }
+        if (!ok) break;
       }
     }
   } else if (warp == 5) {
+    // ---- MMA issuer: accumulator i & 1 for the CTA's i-th tile ----
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16_f32(kGemmBM, kGemmBN, 0);
       bool ok = true;
-      for (int kt = 0; kt < n_k; ++kt) {
-        const int s = kt % kGemmStages;
-        if (!(ok = mbar_wait(bar_full + 8 * s, (kt / kGemmStages) & 1, abort_flag))) break;
+      long long it = 0;
+      int i = 0;
+      for (long long t = blockIdx.x; ok && t < n_tiles; t += gridDim.x, ++i) {
+        const int a = i & 1;
+        if (i >= 2 && !(ok = mbar_wait(bar_acc_empty + 8 * a, (uint32_t)((i >> 1) - 1) & 1, abort_flag))) break;
         tc_fence_after();
-        const uint32_t a = base + s * kGemmStageBytes;
-        mma_ss_4steps(tmem_base, desc_lo(a, 16), desc_lo(a + kGemmABytes, 16), desc_hi_sw128(1024), idesc, kt > 0 ? 1u : 0u);
-        mma_commit(bar_empty + 8 * s);
+        for (int kt = 0; kt < n_k; ++kt, ++it) {
+          const int s = (int)(it % kGemmStages);
+          if (!(ok = mbar_wait(bar_full + 8 * s, (uint32_t)(it / kGemmStages) & 1, abort_flag))) break;
+          tc_fence_after();
+          const uint32_t sa = base + s * kGemmStageBytes;
+          mma_ss_4steps(tmem_base + a * kGemmBN, desc_lo(sa, 16), desc_lo(sa + kGemmABytes, 16), desc_hi_sw128(1024), idesc,
+                        kt > 0 ? 1u : 0u);
+          mma_commit(bar_empty + 8 * s);
+        }
+        if (ok) mma_commit(bar_acc_full + 8 * a);
       }
-      if (ok) mma_commit(bar_acc);
     }
   } else {
     // ---- epilogue: thread = output row = TMEM lane ----
-    bool ok = mbar_wait(bar_acc, 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    int i = 0;
+    for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+      const int a = i & 1;
+      int tm, tn;
+      tile_of(t, tm, tn);
+      bool ok = mbar_wait(bar_acc_full + 8 * a, (uint32_t)(i >> 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
       const long long row = (long long)tm * kGemmBM + warp * 32 + lane;
-      const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+      const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16) + a * kGemmBN;
 #pragma unroll 1
       for (int c = 0; c < kGemmBN / 32; ++c) {
         uint32_t v[32];
@@ -96,13 +127,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (row < M && col0 < N) {
           const long long off = row * N + col0;
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            if (col0 + i < N) {                                  // N is a multiple of 8
+          for (int i8 = 0; i8 < 32; i8 += 8) {
+            if (col0 + i8 < N) {                                 // N is a multiple of 8
               float f[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i + e]);
+              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i8 + e]);
               if (residual != nullptr) {
-                const uint4 r = __ldg(reinterpret_cast<const uint4*>(residual + off + i));
+                const uint4 r = __ldg(reinterpret_cast<const uint4*>(residual + off + i8));
                 const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) { f[2 * e] += __uint_as_float(rw[e] << 16); f[2 * e + 1] += __uint_as_float(rw[e] & 0xffff0000u); }
@@ -113,22 +144,25 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
                 w[e] = *reinterpret_cast<uint32_t*>(&h2);
               }
-              *reinterpret_cast<uint4*>(y + off + i) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(y + off + i8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
       }
+      // the accumulator has been read out: the MMA warp may overwrite it
+      tc_fence_before();
+      mbar_arrive(bar_acc_empty + 8 * a);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_GEMM_SM100, tm, tn);
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_GEMM_SM100, (int)blockIdx.x, 0);
     const uint64_t tw = global_timer_ns();
     while (global_timer_ns() - tw < 200000ull) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, 256); }
+  if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, 512); }
 }
 
 }  // namespace relaxkv
@@ -155,9 +189,13 @@ extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, cons
       return RELAXKV_ERR_CUDA;
     attr_done[dev] = true;
   }
+  static int sm_count[64] = {0};
+  if (sm_count[dev] == 0 && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return RELAXKV_ERR_CUDA;
   const long long tiles_m = (n_rows + kGemmBM - 1) / kGemmBM, tiles_n = (n_out + kGemmBN - 1) / kGemmBN;
   if (tiles_m * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
-  gemm_sm100_kernel<<<(unsigned)(tiles_m * tiles_n), kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
+  const long long grid = std::min<long long>(tiles_m * tiles_n, sm_count[dev]);     // persistent: one CTA per SM
+  gemm_sm100_kernel<<<(unsigned)grid, kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
       tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), st);
   return launch_ok();
 }
