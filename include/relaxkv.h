@@ -295,6 +295,15 @@ relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64
 relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
                               int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream);
 
+/* out = silu(x Wg^T) * (x Wu^T) in one kernel (the MLP's first half): the gate and up projections and the
+ * activation, with one rounding to bf16.  weight_tiled [2 * n_inter, n_in] holds, for every block t of 128
+ * intermediate features, the 128 gate rows Wg[128 t .. 128 t + 127] followed by the 128 up rows Wu[same range]
+ * (a fixed re-ordering of the rows of [Wg; Wu], done once when the weights are loaded), so that a 128 x 256
+ * output tile of the GEMM carries both halves of the same features.  n_inter a multiple of 128.
+ * x [n_rows, n_in], out [n_rows, n_inter]. */
+relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weight_tiled, void* out, int64_t n_rows,
+                                     int32_t n_inter, int32_t n_in, relaxkv_stream stream);
+
 /* Rotary embedding in place, rotate-half convention: pair i < D/2 of each head vector is rotated by
  * positions[row] * theta^(-2i/D).  x [n_rows, n_heads, head_dim]; positions: device int32 [n_rows], the rows'
  * ORIGINAL global positions (Section 3.3: restricting the context does not renumber tokens).  Rotations

@@ -25,7 +25,7 @@ ENTRY_POINTS = (
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_debug_set_attention_splits",
     "relaxkv_list_attention", "relaxkv_cache_attention",
-    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_rope",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_swiglu", "relaxkv_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
 
@@ -285,6 +285,23 @@ def relaxkv_linear(x: torch.Tensor, weight: torch.Tensor, y: torch.Tensor, resid
     """y = x weight^T (+ residual); weight is [n_out, n_in]."""
     _check(lib().relaxkv_linear(_ptr(x), _ptr(weight), _ptr(residual), _ptr(y), ctypes.c_int64(x.shape[0]),
                                 int(weight.shape[0]), int(weight.shape[1]), _stream(stream)), "relaxkv_linear")
+
+
+def tile_gate_up(w_gate_up: torch.Tensor) -> torch.Tensor:
+    """[Wg; Wu] of shape [2 * I, K] -> the row order relaxkv_linear_swiglu reads: per block of 128 features, its gate
+    rows then its up rows.  A weight-loading step (done once), not part of the path."""
+    two_i, k = w_gate_up.shape
+    inter = two_i // 2
+    assert inter % 128 == 0
+    g = w_gate_up[:inter].view(inter // 128, 128, k)
+    u = w_gate_up[inter:].view(inter // 128, 128, k)
+    return torch.cat([g, u], dim=1).reshape(two_i, k).contiguous()
+
+
+def relaxkv_linear_swiglu(x: torch.Tensor, weight_tiled: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    _check(lib().relaxkv_linear_swiglu(_ptr(x), _ptr(weight_tiled), _ptr(out), ctypes.c_int64(x.shape[0]),
+                                       int(weight_tiled.shape[0] // 2), int(weight_tiled.shape[1]), _stream(stream)),
+           "relaxkv_linear_swiglu")
 
 
 def relaxkv_rope(x: torch.Tensor, positions: torch.Tensor, theta: float, stream=None) -> None:

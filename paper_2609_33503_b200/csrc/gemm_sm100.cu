@@ -25,7 +25,7 @@ constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 8 * kGemmBars + 16 + 1
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   long long M, int N, int K, uint16_t* __restrict__ y, const uint16_t* __restrict__ residual,
-                  DeviceStatus* st) {
+                  int swiglu, DeviceStatus* st) {
   const int tiles_m = (int)((M + kGemmBM - 1) / kGemmBM), tiles_n = (N + kGemmBN - 1) / kGemmBN;
   const long long n_tiles = (long long)tiles_m * tiles_n;
   if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;
@@ -118,6 +118,34 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       tc_fence_after();
       const long long row = (long long)tm * kGemmBM + warp * 32 + lane;
       const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16) + a * kGemmBN;
+      if (swiglu) {
+        // the tile's columns are [128 gate | 128 up] of the same 128 intermediate features (weight rows arranged so
+        // by the caller): out[row, tn * 128 + j] = silu(gate_j) * up_j, fp32, one rounding to bf16
+        const int n_inter = N / 2;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t g[32], u[32];
+          tmem_ld32(t_lane + c * 32, g);
+          tmem_ld32(t_lane + 128 + c * 32, u);
+          tmem_wait_ld();
+          const int col0 = tn * 128 + c * 32;
+          if (row < M && col0 < n_inter) {
+            const long long off = row * n_inter + col0;
+#pragma unroll
+            for (int i8 = 0; i8 < 32; i8 += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float g0 = __uint_as_float(g[i8 + 2 * e]), g1 = __uint_as_float(g[i8 + 2 * e + 1]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * __uint_as_float(u[i8 + 2 * e]),
+                                                          g1 / (1.f + __expf(-g1)) * __uint_as_float(u[i8 + 2 * e + 1]));
+                w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(y + off + i8) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else
 #pragma unroll 1
       for (int c = 0; c < kGemmBN / 32; ++c) {
         uint32_t v[32];
@@ -169,11 +197,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 
 using namespace relaxkv;
 
-extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
-                                         int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream_) {
+static relaxkv_status launch_gemm(const void* x, const void* weight, const void* residual, void* y, int64_t n_rows,
+                                  int32_t n_out, int32_t n_in, int swiglu, relaxkv_stream stream_) {
   if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || (residual && !aligned16(residual)))
     return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_out < 8 || n_in < 8 || (n_out % 8) || (n_in % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (swiglu && ((n_out % 256) || residual)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
   CUtensorMap tm_a, tm_b;
   if (!make_map_3d(&tm_a, x, (uint64_t)n_in, (uint64_t)n_rows, 1, (uint64_t)n_in * 2, (uint64_t)n_in * 2 * (uint64_t)n_rows, kGemmBM, 1) ||
@@ -196,6 +225,17 @@ extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, cons
   if (tiles_m * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   const long long grid = std::min<long long>(tiles_m * tiles_n, sm_count[dev]);     // persistent: one CTA per SM
   gemm_sm100_kernel<<<(unsigned)grid, kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
-      tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), st);
+      tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, st);
   return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
+                                         int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream_) {
+  return launch_gemm(x, weight, residual, y, n_rows, n_out, n_in, 0, stream_);
+}
+
+extern "C" relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weight_tiled, void* y, int64_t n_rows,
+                                                int32_t n_inter, int32_t n_in, relaxkv_stream stream_) {
+  if (n_inter < 128 || (n_inter % 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  return launch_gemm(x, weight_tiled, nullptr, y, n_rows, 2 * n_inter, n_in, 1, stream_);
 }

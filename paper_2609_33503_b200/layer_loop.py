@@ -61,7 +61,12 @@ class LayerLoop:
             rec("scatter", lambda: s.scatter(l, caches[l], k, v, n_r[l]))
             rec("o_proj", lambda: B.relaxkv_linear(o.view(n, -1), w["wo"], a, residual=h))
             rec("norm", lambda: B.relaxkv_rmsnorm(a, w["w_post_norm"], x, blk.eps))
-            rec("mlp", lambda: (B.relaxkv_linear(x, w["w_gate_up"], gu), B.relaxkv_swiglu(gu, m)))
+            if blk.inter % 128 == 0:
+                if "w_gate_up_tiled" not in w:          # weight-loading step, once per layer
+                    w["w_gate_up_tiled"] = B.tile_gate_up(w["w_gate_up"])
+                rec("mlp", lambda: B.relaxkv_linear_swiglu(x, w["w_gate_up_tiled"], m))
+            else:
+                rec("mlp", lambda: (B.relaxkv_linear(x, w["w_gate_up"], gu), B.relaxkv_swiglu(gu, m)))
             h_out = self.h_next[:n]
             rec("mlp", lambda: B.relaxkv_linear(m, w["w_down"], h_out, residual=a))
             if l + 1 < L:

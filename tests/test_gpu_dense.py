@@ -169,6 +169,25 @@ def test_whole_repair_loop_with_block_work():
     assert err.mean() <= 1e-2 * scale_ and err.max() <= 0.15 * max(1.0, np.abs(ref).max()), (err.mean(), err.max(), scale_)
 
 
+@pytest.mark.parametrize("M,I,K", [(300, 256, 320), (129, 128, 72), (1000, 1024, 512), (1, 128, 8)])
+def test_linear_swiglu_fused(M, I, K):
+    """Gate and up projections + SwiGLU in one kernel (weights re-ordered per 128-feature block) against the
+    oracle's linear followed by swiglu on the original [gate; up] weights."""
+    x, w = rnd(M, K, seed=4), rnd(2 * I, K, scale=K ** -0.5, seed=5)
+    out = torch.full((M, I), 7.0, dtype=torch.bfloat16, device="cuda")
+    B().relaxkv_linear_swiglu(x, B().tile_gate_up(w), out)
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+    ref = blk.swiglu(blk.linear(blk.f64(bits(x)), blk.f64(bits(w)), None))
+    close(out, ref, abs_floor=2e-3)
+    # the two-kernel route (projection rounded to bf16, then the activation) agrees to a rounding
+    gu = torch.empty(M, 2 * I, dtype=torch.bfloat16, device="cuda")
+    two = torch.empty_like(out)
+    B().relaxkv_linear(x, w, gu)
+    B().relaxkv_swiglu(gu, two)
+    assert float((out.float() - two.float()).abs().max()) <= 2.0 ** -6 * float(two.float().abs().max()) + 1e-2
+
+
 def test_rope_realigns_keys_of_a_moved_chunk():
     """Positional consistency (Section 2): a chunk cached at one offset and placed at another is re-aligned by
     rotating its cached keys by the offset difference.  The keys of a 512-token chunk are rotated at offset
