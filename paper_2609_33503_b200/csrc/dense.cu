@@ -50,6 +50,31 @@ rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, u
   }
 }
 
+// Short rows (a head vector: C <= 256): one warp per row, each lane 8 elements, so the per-head Q/K norm of a
+// [rows, heads, D] tensor is one pass over it.  In place (y == x) is fine: a lane writes what it alone read.
+__global__ void __launch_bounds__(256)
+rmsnorm_short_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y, long long rows,
+                     int C, float eps) {
+  const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const bool mine = lane * 8 < C;
+  float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (mine) unpack8(*reinterpret_cast<const uint4*>(x + row * C + lane * 8), f);
+  float ss = 0.f;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+  ss = warp_reduce_sum(ss);
+  const float inv = rsqrtf(ss / (float)C + eps);
+  if (mine) {
+    float g[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(w + lane * 8)), g);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = f[e] * inv * g[e];
+    *reinterpret_cast<uint4*>(y + row * C + lane * 8) = pack8(f);
+  }
+}
+
 // Rotate-half rotary embedding in place on x [rows, heads, D]; one thread per (row, 8 pairs): the eight
 // (cos, sin) pairs are computed once and applied to every head of the row.
 __global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads, int D, const int* __restrict__ positions,
@@ -156,6 +181,14 @@ extern "C" relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, voi
   if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || !(eps >= 0.f)) return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_cols < 8 || (n_cols % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
+  if (n_cols <= 256) {
+    const long long blocks = (n_rows * 32 + 255) / 256;
+    if (blocks > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+    rmsnorm_short_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(y), n_rows, n_cols, eps);
+    return launch_ok();
+  }
+  if (n_rows > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   rmsnorm_kernel<<<(unsigned)n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(y), n_cols, eps);
   return launch_ok();

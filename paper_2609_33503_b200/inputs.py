@@ -222,14 +222,16 @@ NAMED: Dict[str, object] = {
 
 @dataclasses.dataclass(frozen=True)
 class BlockShape:
-    """Llama-style pre-norm decoder block: hidden size, SwiGLU width, rotary base, RMSNorm epsilon."""
+    """Llama-style pre-norm decoder block: hidden size, SwiGLU width, rotary base, RMSNorm epsilon; `qk_norm`
+    adds the per-head RMSNorm of the projected queries and keys (Qwen3)."""
     hidden: int
     inter: int
     rope_theta: float = 1.0e6
     eps: float = 1.0e-6
+    qk_norm: bool = False
 
 
-QWEN3_14B_BLOCK = BlockShape(hidden=5120, inter=17408)
+QWEN3_14B_BLOCK = BlockShape(hidden=5120, inter=17408, qk_norm=True)
 LLAMA31_8B_BLOCK = BlockShape(hidden=4096, inter=14336, rope_theta=5.0e5, eps=1.0e-5)
 
 
@@ -245,8 +247,11 @@ def block_weights(w: Workload, blk: BlockShape, layer: int, device="cpu") -> Dic
     def gain(n):
         return (1.0 + 0.1 * torch.randn(n, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
 
-    return {"w_in_norm": gain(C), "wq": lin(H * D, C), "wk": lin(Hkv * D, C), "wv": lin(Hkv * D, C), "wo": lin(C, H * D),
-            "w_post_norm": gain(C), "w_gate_up": lin(2 * I, C), "w_down": lin(C, I)}
+    out = {"w_in_norm": gain(C), "wq": lin(H * D, C), "wk": lin(Hkv * D, C), "wv": lin(Hkv * D, C), "wo": lin(C, H * D),
+           "w_post_norm": gain(C), "w_gate_up": lin(2 * I, C), "w_down": lin(C, I)}
+    if blk.qk_norm:
+        out["w_q_norm"], out["w_k_norm"] = gain(D), gain(D)
+    return out
 
 
 def input_representations(w: Workload, blk: BlockShape, req: int, positions: torch.Tensor, device="cpu") -> torch.Tensor:

@@ -1,5 +1,6 @@
 """The repair loop of Algorithm 1 (steps 13-22) with the dense block work included: for every layer the
-active targets run the whole decoder block - RMSNorm, Q/K/V projections, rotary embedding at their original
+active targets run the whole decoder block - RMSNorm, Q/K/V projections, the per-head Q/K norm where the
+model has one, rotary embedding at their original
 positions, sparse-context repair attention, cache update, output projection, MLP - and the hidden rows of
 the targets that stay active are carried to the next layer.  This module only sequences calls of the C ABI
 (`binding`) over torch buffers; every operation runs in the CUDA kernels.
@@ -38,6 +39,7 @@ class LayerLoop:
         s, blk = self.s, self.blk
         n_u, n_r = s.counts()
         L = s.n_layers
+        D = s.shape.c.head_dim
 
         def rec(name, fn):
             if events is None:
@@ -55,6 +57,9 @@ class LayerLoop:
             rec("norm", lambda: B.relaxkv_rmsnorm(h, w["w_in_norm"], x, blk.eps))
             rec("qkv_proj", lambda: (B.relaxkv_linear(x, w["wq"], q.view(n, -1)), B.relaxkv_linear(x, w["wk"], k.view(n, -1)),
                                      B.relaxkv_linear(x, w["wv"], v.view(n, -1))))
+            if "w_q_norm" in w:                       # per-head RMSNorm of the projected queries and keys, in place
+                rec("norm", lambda: (B.relaxkv_rmsnorm(q.view(-1, D), w["w_q_norm"], q.view(-1, D), blk.eps),
+                                     B.relaxkv_rmsnorm(k.view(-1, D), w["w_k_norm"], k.view(-1, D), blk.eps)))
             rec("rope", lambda: (B.relaxkv_target_positions(s.shape, s.u_pos, s.u_cu, s.r_rank, s.r_cu_layer(l), n_r[l], pos),
                                  B.relaxkv_rope(q, pos, blk.rope_theta), B.relaxkv_rope(k, pos, blk.rope_theta)))
             rec("attention", lambda: s.attention(l, caches[l], q, k, v, o, n_r[l], n_u))

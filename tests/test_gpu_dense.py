@@ -53,6 +53,11 @@ def test_rmsnorm_rope_swiglu():
     y = torch.empty_like(x)
     B().relaxkv_rmsnorm(x, w, y, 1e-6)
     close(y, blk.rmsnorm(blk.f64(bits(x)), blk.f64(bits(w)), 1e-6), abs_floor=1e-3)
+    for C in (64, 128, 256):                                    # head vectors: one warp per row, also in place
+        xs, ws = rnd(53 * 5, C, seed=8, scale=2.0), rnd(C, seed=9)
+        ref = blk.rmsnorm(blk.f64(bits(xs)), blk.f64(bits(ws)), 1e-6)
+        B().relaxkv_rmsnorm(xs, ws, xs, 1e-6)
+        close(xs, ref, abs_floor=1e-3)
     for D in (64, 128):
         q = rnd(53, 5, D, seed=6)
         pos = torch.tensor(np.random.default_rng(0).integers(0, 66000, size=53).astype(np.int32)).cuda()
@@ -114,7 +119,7 @@ def test_whole_repair_loop_with_block_work():
     from tests.harness import Case
     w = inputs.Workload("block", 3, 4, 2, 64, 64, (600, 380), (8, 5), 0.15, base_seed=3,
                         planted_chunks=((2, 7), (1,)), variant="calibrated")
-    blkshape = inputs.BlockShape(hidden=256, inter=512, rope_theta=1.0e4, eps=1.0e-5)
+    blkshape = inputs.BlockShape(hidden=256, inter=512, rope_theta=1.0e4, eps=1.0e-5, qk_norm=True)
     case = Case(w)
     s = case.make_session()
     s.build_active_sets(case.anchors_tensor())
@@ -145,6 +150,8 @@ def test_whole_repair_loop_with_block_work():
             q = bf16_round(blk.linear(x, W["wq"])).reshape(n, H, D)
             k = bf16_round(blk.linear(x, W["wk"])).reshape(n, Hkv, D)
             v = bf16_round(blk.linear(x, W["wv"])).reshape(n, Hkv, D)
+            q = bf16_round(blk.rmsnorm(q.reshape(n * H, D), W["w_q_norm"], blkshape.eps)).reshape(n, H, D)
+            k = bf16_round(blk.rmsnorm(k.reshape(n * Hkv, D), W["w_k_norm"], blkshape.eps)).reshape(n, Hkv, D)
             q, k = bf16_round(blk.rope(q, pos, blkshape.rope_theta)), bf16_round(blk.rope(k, pos, blkshape.rope_theta))
             o, _ = orc.repair_attention(case.req_k(l, b), case.req_v(l, b), to_bits(q), to_bits(k), to_bits(v), sets.u_pos,
                                         sets.ranks(l), case.scale)
