@@ -37,7 +37,8 @@ struct AttnSmem {
   static constexpr int kQ = 0;                                  // two query tiles
   static constexpr int kKV = kQ + 2 * kTileBytes;               // ring of kRing K/V tiles
   static constexpr int kBar = kKV + kRing * kTileBytes;         // mbarriers (8 B each)
-  static constexpr int kNumBars = 1 + 8 + 2 * kRing;
+  static constexpr int kPairBars = 3;                           // (V_j, K_{j+1}) pairs in flight: full and empty barriers
+  static constexpr int kNumBars = 1 + 8 + 2 * kPairBars;
   static constexpr int kMisc = kBar + 8 * kNumBars;             // tmem address, abort flag
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                // slack to align the base to 1024 B
@@ -130,8 +131,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_pfull = bar0 + 24;         // [2] first 64 keys of P ready
   const uint32_t bar_pfull_hi = bar0 + 40;      // [2] last 64 keys of P ready
   const uint32_t bar_ofinal = bar0 + 56;        // [2]
-  const uint32_t bar_full = bar0 + 72;          // [kRing]
-  const uint32_t bar_empty = bar_full + 8 * kRing;
+  const uint32_t bar_full = bar0 + 72;          // [kPairBars] pair p = (V_{p-1}, K_p) has landed
+  const uint32_t bar_empty = bar_full + 8 * L::kPairBars;   // [kPairBars] pair p has been consumed by both tiles
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
 
@@ -140,7 +141,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
     for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_pfull_hi + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
-    for (int s = 0; s < kRing; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -177,14 +178,27 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int hf = 0; hf < kHalves; ++hf)
           tma_load_3d(q_smem + (x * kHalves + hf) * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G,
                       (int)(q_row_base + x * tile_targets));
-      for (int u = 0; u < 2 * n_my_max; ++u) {                // u = 2*j + (0: K, 1: V), j counted from j0
+      // The tiles travel in the order K_0 V_0 K_1 V_1 ... through the ring slots u % kRing (u = 2j for K_j, 2j + 1
+      // for V_j; j counted from j0).  They are signalled in PAIRS p = (V_{p-1}, K_p): step j of the MMA warp needs
+      // exactly pair j + 1 (V_j for P V, K_{j+1} for the next Q K^T), so it waits once and frees once per step.
+      auto load_tile = [&](int u, uint32_t bar) {
         const int s = u % kRing;
-        if (u >= kRing && !mbar_wait(bar_empty + 8 * s, ((u / kRing) - 1) & 1, abort_flag)) break;
         const int row = (int)(ctx_base + (long long)(j0 + (u >> 1)) * kBN);
         const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
-        mbar_expect_tx(bar_full + 8 * s, L::kTileBytes);
         for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar_full + 8 * s, hf * 64, hd, row);
+          tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar, hf * 64, hd, row);
+      };
+      for (int pr = 0; pr <= n_my_max; ++pr) {                  // pair pr: V_{pr-1} (if pr > 0) and K_pr (if pr < n)
+        const uint32_t bar = bar_full + 8 * (pr % L::kPairBars);
+        const bool has_v = pr > 0, has_k = pr < n_my_max;
+        // slot of V_{pr-1} was last used by K_{pr-3} (pair pr-3), slot of K_pr by V_{pr-3} (pair pr-2)
+        if (pr >= 3 && !mbar_wait(bar_empty + 8 * ((pr - 3) % L::kPairBars), (uint32_t)((pr - 3) / L::kPairBars) & 1, abort_flag)) break;
+        mbar_expect_tx(bar, (uint32_t)((has_v ? L::kTileBytes : 0) + (has_k ? L::kTileBytes : 0)));
+        if (has_v) load_tile(2 * pr - 1, bar);
+        if (has_k) {
+          if (pr >= 3 && !mbar_wait(bar_empty + 8 * ((pr - 2) % L::kPairBars), (uint32_t)((pr - 2) / L::kPairBars) & 1, abort_flag)) break;
+          load_tile(2 * pr, bar);
+        }
       }
     }
   } else if (warp == 9) {
@@ -194,21 +208,15 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       // S_x = Q_x K_j^T  -> bar_sfull[x]
-      // (a successful mbarrier wait costs the issuing thread ~150 cycles, so a tile that is known to be
-      //  in shared memory - the other query tile already waited for it - is not waited for again)
-      auto issue_qk = [&](int x, int j, bool wait_tile) -> bool {
-        const int u = 2 * j, s = u % kRing;
-        if (wait_tile && !mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
-        tc_fence_after();
+      auto issue_qk = [&](int x, int j) {
+        const int s = (2 * j) % kRing;
         mma_ss_kloop<kHalves>(tmem_base + x * 128, desc_lo(q_smem + x * L::kTileBytes, 16),
                               desc_lo(kv_smem + s * L::kTileBytes, 16), desc_hi_sw128(1024), idesc_qk);
         mma_commit(bar_sfull + 8 * x);
-        return true;
       };
       // O_x += P_x V_j   (P_x read from TMEM where the softmax warps left it, over S_x)
-      auto issue_pv = [&](int x, int j, bool wait_tile) -> bool {
-        const int u = 2 * j + 1, s = u % kRing;
-        if (wait_tile && !mbar_wait(bar_full + 8 * s, (u / kRing) & 1, abort_flag)) return false;
+      auto issue_pv = [&](int x, int j) -> bool {
+        const int s = (2 * j + 1) % kRing;
         if (!mbar_wait(bar_pfull + 8 * x, j & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t v_lo = desc_lo(kv_smem + s * L::kTileBytes, kHalfBytes);
@@ -220,21 +228,27 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (j == n_my[x] - 1) mma_commit(bar_ofinal + 8 * x);
         return true;
       };
-      if (ok && n_my[0] > 0) ok = issue_qk(0, 0, true);
-      if (ok && n_my[1] > 0) ok = issue_qk(1, 0, n_my[0] == 0);
-      if (ok) mma_commit(bar_empty + 8 * 0);                   // K_0's buffer: free once both S tiles are done
-      for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0
-        const bool a_pv = j < n_my[0], a_qk = j + 1 < n_my[0];
-        if (a_pv) {
-          if (!(ok = issue_pv(0, j, true))) break;
-          if (a_qk && !(ok = issue_qk(0, j + 1, true))) break;
+      // pair 0 = K_0 alone
+      if (ok) ok = mbar_wait(bar_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        if (n_my[0] > 0) issue_qk(0, 0);
+        if (n_my[1] > 0) issue_qk(1, 0);
+        mma_commit(bar_empty);
+      }
+      for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0; this step consumes pair j + 1
+        const int pr = j + 1;
+        if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
+        tc_fence_after();
+        if (j < n_my[0]) {
+          if (!(ok = issue_pv(0, j))) break;
+          if (j + 1 < n_my[0]) issue_qk(0, j + 1);
         }
         if (j < n_my[1]) {
-          if (!(ok = issue_pv(1, j, !a_pv))) break;
+          if (!(ok = issue_pv(1, j))) break;
+          if (j + 1 < n_my[1]) issue_qk(1, j + 1);
         }
-        mma_commit(bar_empty + 8 * ((2 * j + 1) % kRing));     // V_j
-        if (j + 1 < n_my[1] && !(ok = issue_qk(1, j + 1, !a_qk))) break;
-        if (j + 1 < n_my_max) mma_commit(bar_empty + 8 * ((2 * j + 2) % kRing));   // K_{j+1}
+        mma_commit(bar_empty + 8 * (pr % L::kPairBars));        // V_j and K_{j+1}: free once both tiles are through
       }
     }
   }
