@@ -10,8 +10,13 @@
 // A CTA runs TWO such query tiles (A, B) in ping-pong: while the softmax warps of one tile work, the
 // tensor pipe runs the other tile's MMAs; both tiles share every K/V tile staged in shared memory.
 // Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = query row = TMEM
-// lane), warp 8 TMA producer, warp 9 MMA issuer and TMEM owner.  Every wait is bounded; an expired wait raises the block's abort
-// flag, records RELAXKV_ERR_TIMEOUT in the device status word and the block tears down normally.
+// lane), warp 8 TMA producer, warp 9 MMA issuer and TMEM owner.  K/V tiles move through a 5-slot ring in the
+// order K_0 V_0 K_1 V_1 ... and are signalled in pairs (V_j, K_{j+1}) - what step j of the MMA warp consumes.
+// When a call has too few query tiles to fill the GPU, grid.y splits every pair's context; the blocks leave
+// normalised partial results that combine_splits_kernel merges by their log-sum-exp.  The K/V tensor maps
+// cover either the materialised mixed context (the repair calls) or the cache itself (relaxkv_cache_attention).
+// Every wait is bounded; an expired wait raises the block's abort flag, records RELAXKV_ERR_TIMEOUT in the
+// device status word and the block tears down normally.
 #include "attention_common.cuh"
 #include "sm100_ptx.cuh"
 #include <algorithm>
