@@ -231,6 +231,8 @@ def run_gpu(args):
         raise SystemExit("librelaxkv.so is missing: run `python __graft_entry__.py` first (no CPU fallback exists)")
     w = make_workload(args)
     peaks = load_peaks()
+    if args.sm_pairs:
+        B.relaxkv_debug_set_attention_sm_pairs(True)
     job = GpuJob(w, device)
     mode = B.CTX_FULL_PREFIX if args.full_prefix else B.CTX_UNION
     for _ in range(args.warmup):
@@ -644,6 +646,7 @@ def main():
                          "rotary embedding, MLP with synthetic weights); prints its own JSON line")
     ap.add_argument("--query-attention", action="store_true",
                     help="time the user query's prefill rows and a decode step over the context cache (same kernel, context split)")
+    ap.add_argument("--sm-pairs", action="store_true", help="run the attention on the opt-in SM-pair kernel (cta_group::2)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows", type=int, default=256)

@@ -371,6 +371,14 @@ relaxkv_status relaxkv_cache_attention(
 relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits);
 
 /*
+ * Test utility (the paper has no counterpart).  on != 0 makes every later attention call of this process with
+ * head_dim 128 run the SM-pair variant of the kernel (clusters of two thread blocks whose tensor cores are driven
+ * by one instruction stream, each block staging half of every K/V tile); 0 restores the single-block kernel, the
+ * default (it measures faster).  Results agree within the attention tolerance.
+ */
+relaxkv_status relaxkv_debug_set_attention_sm_pairs(int32_t on);
+
+/*
  * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on
  * a barrier nothing will ever complete.  The wait gives up after its limit (0.4 s), the kernel ends
  * normally and RELAXKV_ERR_TIMEOUT is recorded in the device status word - the same path a stuck

@@ -230,6 +230,90 @@ __device__ __forceinline__ void mma_ts_4steps(uint32_t d_tmem, uint32_t a_tmem, 
       "}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first) : "memory");
 }
 
+// ---- CTA pairs (cta_group::2): one MMA instruction drives the tensor cores of two SMs ----------------------
+// A cluster of two CTAs; rank 0 (the leader) issues.  For M = 256 each CTA supplies 128 rows of A (its own shared
+// memory or TMEM, same offsets in both), HALF of B's N rows from its own shared memory, and receives its 128 rows
+// of D (all N columns) in its own TMEM.  alloc / dealloc are executed by one warp of EACH CTA.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {      // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cta address -> the same offset in CTA `rank` of the cluster (a shared::cluster address)
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// bounded wait on a barrier that also receives arrivals from the other CTA of the cluster
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if ((it & 63u) == 0u && global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+  }
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {   // whole warp, in each CTA
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// One arrival on the barrier at this offset in every CTA of `mask`, once all MMAs issued so far have completed.
+// (A commit with cluster multicast, not a multicast copy: nothing is loaded.)
+__device__ __forceinline__ void mma_commit2_mc(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+#define RELAXKV_MMA2_SS_STEP(AOFF, BOFF, PRED)                                               \
+  "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                                  \
+  "mov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"                                           \
+  "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, " #PRED ";\n\t"
+// D[tmem] = A[smem] * B[smem] over K = 128 (two 64-element halves; A's halves 16 KB apart, B's 8 KB: this CTA's
+// 64 of the tile's 128 N rows): the first MMA overwrites D.
+__device__ __forceinline__ void mma2_ss_kloop(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      RELAXKV_MMA2_SS_STEP(0, 0, p0) RELAXKV_MMA2_SS_STEP(2, 2, p1) RELAXKV_MMA2_SS_STEP(4, 4, p1) RELAXKV_MMA2_SS_STEP(6, 6, p1)
+      RELAXKV_MMA2_SS_STEP(1024, 512, p1) RELAXKV_MMA2_SS_STEP(1026, 514, p1) RELAXKV_MMA2_SS_STEP(1028, 516, p1)
+      RELAXKV_MMA2_SS_STEP(1030, 518, p1)
+      "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+}
+#define RELAXKV_MMA2_TS_STEP(AOFF, BOFF, PRED)                                               \
+  "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                                  \
+  "mov.b64 db, {tb, %3};\n\t"                                                                  \
+  "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %4, " #PRED ";\n\t"
+// D[tmem] (+)= A[tmem] * B[smem] for four K steps of 16: A advances 8 columns, B (MN-major) 2048 bytes per step.
+__device__ __forceinline__ void mma2_ts_4steps(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                               uint32_t acc_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      RELAXKV_MMA2_TS_STEP(0, 0, p0) RELAXKV_MMA2_TS_STEP(8, 128, p1) RELAXKV_MMA2_TS_STEP(16, 256, p1) RELAXKV_MMA2_TS_STEP(24, 384, p1)
+      "}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first) : "memory");
+}
+
 // ---- descriptors ------------------------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle, tiles whose 8-row groups are 1024 bytes apart.
 //   K-major operand  (rows of 64 bf16 = 128 B):       lbo ignored (1),  sbo = 1024

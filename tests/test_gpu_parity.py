@@ -269,6 +269,25 @@ def test_context_split_matches_oracle(case, n_splits):
         B().relaxkv_debug_set_attention_splits(0)
 
 
+@pytest.mark.parametrize("n_splits", [0, 3])
+def test_sm_pair_kernel_matches_oracle(case, n_splits):
+    """The opt-in SM-pair variant (clusters of two blocks, one MMA instruction stream for both SMs, half of every
+    K/V tile per block) against the oracle, both context modes, with and without a forced context split; an odd
+    number of tile pairs leaves the last cluster's second block without targets."""
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    B().relaxkv_debug_set_attention_sm_pairs(True)
+    B().relaxkv_debug_set_attention_splits(n_splits)
+    try:
+        for l in range(case.w.n_layers):
+            for full_prefix in (False, True):
+                out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
+                check_attention(case, l, out, lse, full_prefix)
+    finally:
+        B().relaxkv_debug_set_attention_splits(0)
+        B().relaxkv_debug_set_attention_sm_pairs(False)
+
+
 def test_attention_orders_agree_and_is_deterministic(case):
     """Update-then-attend from the cache equals mix-then-attend (Algorithm 1's order), bit for bit;
     two runs give identical bits."""
