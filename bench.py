@@ -231,8 +231,8 @@ def run_gpu(args):
         raise SystemExit("librelaxkv.so is missing: run `python __graft_entry__.py` first (no CPU fallback exists)")
     w = make_workload(args)
     peaks = load_peaks()
-    if args.sm_pairs:
-        B.relaxkv_debug_set_attention_sm_pairs(True)
+    if args.attn_variant:
+        B.relaxkv_debug_set_attention_variant(args.attn_variant)
     job = GpuJob(w, device)
     mode = B.CTX_FULL_PREFIX if args.full_prefix else B.CTX_UNION
     for _ in range(args.warmup):
@@ -646,7 +646,8 @@ def main():
                          "rotary embedding, MLP with synthetic weights); prints its own JSON line")
     ap.add_argument("--query-attention", action="store_true",
                     help="time the user query's prefill rows and a decode step over the context cache (same kernel, context split)")
-    ap.add_argument("--sm-pairs", action="store_true", help="run the attention on the opt-in SM-pair kernel (cta_group::2)")
+    ap.add_argument("--attn-variant", type=int, default=0, choices=[0, 1, 2],
+                    help="attention kernel for head_dim 128: 0 two tiles per block (default), 1 SM pairs, 2 one tile with split keys")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows", type=int, default=256)

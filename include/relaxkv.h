@@ -371,12 +371,15 @@ relaxkv_status relaxkv_cache_attention(
 relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits);
 
 /*
- * Test utility (the paper has no counterpart).  on != 0 makes every later attention call of this process with
- * head_dim 128 run the SM-pair variant of the kernel (clusters of two thread blocks whose tensor cores are driven
- * by one instruction stream, each block staging half of every K/V tile); 0 restores the single-block kernel, the
- * default (it measures faster).  Results agree within the attention tolerance.
+ * Test utility (the paper has no counterpart).  Chooses the kernel every later attention call of this process
+ * with head_dim 128 runs (head_dim 64 always runs variant 0); results agree within the attention tolerance.
+ *   0  two query tiles per thread block in ping-pong (default)
+ *   1  SM pairs: clusters of two blocks whose tensor cores are driven by one instruction stream, each block
+ *      staging half of every K/V tile
+ *   2  one query tile per block, S and P double-buffered in tensor memory, the two softmax warpgroups splitting
+ *      the keys of every tile
  */
-relaxkv_status relaxkv_debug_set_attention_sm_pairs(int32_t on);
+relaxkv_status relaxkv_debug_set_attention_variant(int32_t variant);
 
 /*
  * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on

@@ -881,6 +881,395 @@ attention_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __gr
   }
 }
 
+// ---- one query tile per CTA, S and P double-buffered, the two softmax warpgroups split the KEYS of every tile ---------
+// TMEM: S0 | S1 (2 x 128 columns), O (128), P0 | P1 (2 x 64): with P out of S's columns and a second S buffer the MMA
+// warp issues Q K^T of step j + 1 before P V of step j, so a tile's softmax never waits for its own MMAs (in the
+// two-tile kernel above S and P share columns and every step is a dependency chain).  Thread = (query row, key half):
+// warpgroup h handles keys [64 h, 64 h + 64) of every tile; the two halves of a row agree on the reference exponent
+// through shared memory (one named barrier per step), keep partial row sums, and each rescales half of O's columns.
+struct SplitSmem {
+  static constexpr int kQTileBytes = 2 * kHalfBytes;
+  static constexpr int kTileBytes = 2 * kHalfBytes;               // a whole K or V tile
+  static constexpr int kPairBars = 3;
+  static constexpr int kRing = 2 * kPairBars;
+  static constexpr int kQ = 0;
+  static constexpr int kKV = kQ + kQTileBytes;
+  static constexpr int kXch = kKV + kRing * kTileBytes;           // float [2][128]: row maxima / row sums of the halves
+  static constexpr int kBar = kXch + 2 * 128 * 4;
+  static constexpr int kNumBars = 1 + 2 + 2 + 2 + 2 + 1 + 2 * kPairBars;   // q, sfull, sfree, pfull, pvdone, ofinal, full, empty
+  static constexpr int kMisc = kBar + 8 * kNumBars;
+  static constexpr int kTotal = kMisc + 16;
+  static constexpr int kDynamic = kTotal + 1024;
+};
+
+__device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_split_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
+                             int mode, int allow_empty, int head_inner, int dense_ctx, int H, int Hkv, int tile_targets, float scale_log2,
+                             const int* __restrict__ u_pos, const int* __restrict__ u_cu,
+                             const int* __restrict__ r_rank, const int* __restrict__ r_cu,
+                             long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
+                             float* __restrict__ part_o, float* __restrict__ part_lse, DeviceStatus* st) {
+  using L = SplitSmem;
+  constexpr int D = 128;
+  constexpr int kHalves = 2;
+  constexpr uint32_t kTmemCols = 512;
+  constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
+
+  // ---- which query tile: rt.tile_cu counts TILES per request (host bounds), walked from the end of the target list ----
+  const int B = rt.n_req;
+  const int G = H / Hkv;
+  const int n_tiles_total = rt.tile_cu[B];
+  const int hd = head_inner ? (int)(blockIdx.x % Hkv) : (int)(blockIdx.x / n_tiles_total);
+  const int tt = head_inner ? (int)(blockIdx.x / Hkv) : (int)(blockIdx.x - hd * n_tiles_total);
+  const int b = find_segment(rt.tile_cu, B, tt);
+  const int t_rev = tt - rt.tile_cu[b];
+  const int nr = r_cu[b + 1] - r_cu[b];
+  const int nu = dense_ctx ? rt.ctx_len[b] : (u_cu[b + 1] - u_cu[b]);
+  const int n_tiles_true = (nr + tile_targets - 1) / tile_targets;
+  if (t_rev >= n_tiles_true) return;
+  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b])) {
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
+    return;
+  }
+  if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;   // drain after a timeout
+  const int tile = n_tiles_true - 1 - t_rev;
+  const int rho0 = tile * tile_targets;
+  const int ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
+  const long long ctx_base = dense_ctx ? rt.tok_off[b] : ((mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b]);
+  const long long q_row_base = (long long)(r_cu[b] - r_cu[0]) + rho0;
+  const int n_valid = max(0, min(tile_targets, nr - rho0));
+  int n_kv = 0;
+  {
+    const int c = r_rank[r_cu[b] + rho0 + n_valid - 1];
+    const int cc = min(max(c, 0), max(nu - 1, 0));
+    int lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[u_cu[b] + cc];
+    lim_last = min(max(lim_last, 0), ctx_len_b - 1);
+    n_kv = lim_last / kBN + 1;
+  }
+  const int n_splits = (int)gridDim.y, split = (int)blockIdx.y;
+  const int chunk = (n_kv + n_splits - 1) / n_splits;
+  const int j0 = split * chunk;
+  const int n_my = max(0, min(n_kv, j0 + chunk) - j0);
+  if (n_my == 0) {                            // nothing of this tile's context falls into this split
+    if (n_splits > 1 && threadIdx.x < kBM) {
+      const int row = threadIdx.x, t_local = row / G;
+      if (row < tile_targets * G && t_local < n_valid)
+        part_lse[((long long)split * n_target_rows + q_row_base + t_local) * H + hd * G + (row - t_local * G)] = -INFINITY;
+    }
+    return;
+  }
+
+  // ---- shared memory ----
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_smem = base + L::kQ, kv_smem = base + L::kKV;
+  float* xch = reinterpret_cast<float*>(base_ptr + L::kXch);
+  const uint32_t bar0 = base + L::kBar;
+  const uint32_t bar_q = bar0;
+  const uint32_t bar_sfull = bar0 + 8;          // [2] S buffer written
+  const uint32_t bar_sfree = bar0 + 24;         // [2] S buffer read into registers by all 256 softmax threads
+  const uint32_t bar_pfull = bar0 + 40;         // [2] P buffer written
+  const uint32_t bar_pvdone = bar0 + 56;        // [2] P V of the step that used this P buffer has completed
+  const uint32_t bar_ofinal = bar0 + 72;
+  const uint32_t bar_full = bar0 + 80;          // [kPairBars] pair p = (V_{p-1}, K_p) has landed
+  const uint32_t bar_empty = bar_full + 8 * L::kPairBars;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_sfree + 8 * x, 256); mbar_init(bar_pfull + 8 * x, 256); mbar_init(bar_pvdone + 8 * x, 1);
+    }
+    mbar_init(bar_ofinal, 1);
+    for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 9) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols); tmem_relinquish(); }
+  {
+    const int used = tile_targets * G, n_pad = kBM - used;      // rows no (target, head) pair fills: zero them
+    for (int i = threadIdx.x; i < n_pad * 8 * kHalves; i += kAttnThreads) {
+      const int piece = i & 7, r = (i >> 3) % n_pad, hf = (i >> 3) / n_pad;
+      *reinterpret_cast<uint4*>(base_ptr + L::kQ + hf * kHalfBytes + (used + r) * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp >= 8) {
+  reg_dealloc<56>();
+  if (warp == 8) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+      mbar_expect_tx(bar_q, (uint32_t)(kHalves * tile_targets * G * 128));
+      for (int hf = 0; hf < kHalves; ++hf)
+        tma_load_3d(q_smem + hf * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G, (int)q_row_base);
+      // tiles in the order K_0 V_0 K_1 V_1 ... through ring slots u % kRing, signalled in pairs p = (V_{p-1}, K_p)
+      auto load_tile = [&](int u, uint32_t bar) {
+        const int s = u % L::kRing;
+        const int row = (int)(ctx_base + (long long)(j0 + (u >> 1)) * kBN);
+        const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
+        for (int hf = 0; hf < kHalves; ++hf)
+          tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar, hf * 64, hd, row);
+      };
+      for (int pr = 0; pr <= n_my; ++pr) {
+        const uint32_t bar = bar_full + 8 * (pr % L::kPairBars);
+        const bool has_v = pr > 0, has_k = pr < n_my;
+        if (pr >= L::kPairBars &&
+            !mbar_wait(bar_empty + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(bar, (uint32_t)((has_v ? L::kTileBytes : 0) + (has_k ? L::kTileBytes : 0)));
+        if (has_v) load_tile(2 * pr - 1, bar);
+        if (has_k) load_tile(2 * pr, bar);
+      }
+    }
+  } else if (warp == 9) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(kBM, kBN, 0);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      auto issue_qk = [&](int j) {                              // S_{j & 1} = Q K_j^T
+        const int s = (2 * j) % L::kRing;
+        mma_ss_kloop<kHalves>(tmem_base + kColS + (j & 1) * 128, desc_lo(q_smem, 16), desc_lo(kv_smem + s * L::kTileBytes, 16),
+                              desc_hi_sw128(1024), idesc_qk);
+        mma_commit(bar_sfull + 8 * (j & 1));
+      };
+      if (ok) ok = mbar_wait(bar_full, 0, abort_flag);          // pair 0 = K_0 alone
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0);
+        mma_commit(bar_empty);
+      }
+      for (int j = 0; ok && j < n_my; ++j) {                    // this step consumes pair j + 1 = (V_j, K_{j+1})
+        const int pr = j + 1;
+        if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
+        if (j + 1 < n_my) {
+          // S buffer (j + 1) & 1 was last read by the softmax of step j - 1
+          if (j >= 1 && !(ok = mbar_wait(bar_sfree + 8 * ((j + 1) & 1), (uint32_t)((j - 1) >> 1) & 1, abort_flag))) break;
+          tc_fence_after();
+          issue_qk(j + 1);
+        }
+        // O += P_j V_j   (P buffer j & 1)
+        if (!(ok = mbar_wait(bar_pfull + 8 * (j & 1), (uint32_t)(j >> 1) & 1, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t v_lo = desc_lo(kv_smem + ((2 * j + 1) % L::kRing) * L::kTileBytes, kHalfBytes);
+        const uint32_t t_p = tmem_base + kColP + (j & 1) * 64;
+        mma_ts_4steps(tmem_base + kColO, t_p, v_lo, desc_hi_sw128(1024), idesc_pv, j > 0 ? 1u : 0u);
+        mma_ts_4steps(tmem_base + kColO, t_p + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
+        mma_commit(bar_pvdone + 8 * (j & 1));
+        if (j == n_my - 1) mma_commit(bar_ofinal);
+        mma_commit(bar_empty + 8 * (pr % L::kPairBars));
+      }
+    }
+  }
+  } else {
+    reg_alloc<224>();
+    // ================= softmax + epilogue: thread = (query row = TMEM lane, key half h) =================
+    const int h = warp >> 2;
+    const int row = threadIdx.x & 127;
+    const int t_local = row / G, j_head = row - t_local * G;
+    const bool row_valid = (row < tile_targets * G) && (t_local < n_valid);
+    int limit = 0;
+    bool row_empty = false;
+    if (row_valid) {
+      const int c = r_rank[r_cu[b] + rho0 + t_local];
+      if (c == -1 && allow_empty) {
+        row_empty = true;
+      } else if (c < 0 || c >= nu) {
+        if (h == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
+      } else {
+        limit = (mode == RELAXKV_CTX_UNION) ? c : u_pos[u_cu[b] + c];
+        if (limit < 0 || limit >= ctx_len_b) { if (h == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, limit, ctx_len_b); limit = 0; }
+      }
+    }
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_o = lane_base + kColO + h * 64;             // this thread's half of the row's O columns
+    float m = -INFINITY, z = 0.f;                               // z: this half's partial row sum
+    // Every softmax thread runs every step's two named barriers, whatever happens: a warp whose bounded wait gave up
+    // (`dead`) only skips the work between them, so the unbounded bar.sync can never be left short of arrivals.
+    bool dead = false;
+    for (int j = 0; j < n_my; ++j) {
+      const int buf = j & 1;
+      uint32_t s[64];
+      float mx_half = -INFINITY;
+      if (!dead) {
+        bool ok = mbar_wait(bar_sfull + 8 * buf, (uint32_t)(j >> 1) & 1, abort_flag);
+        dead = !__all_sync(0xffffffffu, ok);
+      }
+      if (!dead) {
+      tc_fence_after();
+      tmem_ld32(lane_base + kColS + buf * 128 + h * 64, &s[0]);
+      tmem_ld32(lane_base + kColS + buf * 128 + h * 64 + 32, &s[32]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(bar_sfree + 8 * buf);                         // the MMA warp may overwrite this S buffer
+      const int col0 = (j0 + j) * kBN + h * 64;
+      if (col0 + 63 > limit) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
+      }
+      float mx8[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
+#pragma unroll
+      for (int i = 8; i + 16 <= 64; i += 16) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mx8[e] = fmax3(mx8[e], __uint_as_float(s[i + e]), __uint_as_float(s[i + 8 + e]));
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[56 + e]));
+      mx_half = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                      fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+      // the two halves of a row agree on the tile's maximum (same value, same decisions in both)
+      xch[h * 128 + row] = mx_half;
+      }
+      named_bar_sync(1, 256);
+      if (!dead) {
+      const float mx = fmaxf(mx_half, xch[(1 - h) * 128 + row]);
+      const float m_new = mx * scale_log2;
+      if (j == 0) {
+        m = fmaxf(m_new, -1.0e30f);
+      } else {
+        const bool need = m_new > m + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {
+          // O must hold every product up to step j - 1 before it is rescaled (Q K^T runs ahead of P V here)
+          bool ok = mbar_wait(bar_pvdone + 8 * ((j - 1) & 1), (uint32_t)((j - 1) >> 1) & 1, abort_flag);
+          dead = !__all_sync(0xffffffffu, ok);
+          if (!dead) {
+            tc_fence_after();
+            float alpha = 1.f;
+            if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              uint32_t o[32];
+              tmem_ld32(t_o + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st32(t_o + c * 32, o);
+            }
+            tmem_wait_st();
+          }
+        }
+      }
+      }
+      // the second named barrier of the step: nobody overwrites xch before both halves have read it
+      named_bar_sync(2, 256);
+      // P buffer `buf` was last read by P V of step j - 2
+      if (!dead && j >= 2) {
+        bool ok = mbar_wait(bar_pvdone + 8 * buf, (uint32_t)((j - 2) >> 1) & 1, abort_flag);
+        dead = !__all_sync(0xffffffffu, ok);
+      }
+      if (!dead) {
+      float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
+      const float neg_m = -m;
+      const uint32_t t_p = lane_base + kColP + buf * 64 + h * 32;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+          float x[8], p[8];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2)
+            fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
+                 scale_log2, neg_m, neg_m);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
+          add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
+          add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(p[e], p[e + 1]);
+            pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+        }
+        tmem_st16(t_p + c * 16, pk);
+      }
+      z += (zs0 + zs1) + (zs2 + zs3);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_pfull + 8 * buf);
+      }
+    }
+    if (!dead) {
+      bool ok = mbar_wait(bar_ofinal, 0, abort_flag);
+      dead = !__all_sync(0xffffffffu, ok);
+    }
+    // total row sum = the two halves' partial sums
+    xch[h * 128 + row] = z;
+    named_bar_sync(1, 256);
+    if (!dead) {
+      tc_fence_after();
+      const float z_row = z + xch[(1 - h) * 128 + row];
+      const bool none = row_empty || !(z_row > 0.f);
+      const float inv = none ? 0.f : 1.f / z_row;
+      const float lse = none ? -INFINITY : (m + log2f(z_row)) * kLn2A;
+      const long long orow = q_row_base + t_local;
+      const long long slot = ((long long)split * n_target_rows + orow) * H + hd * G + j_head;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t o[32];
+        tmem_ld32(t_o + c * 32, o);
+        tmem_wait_ld();
+        if (row_valid) {
+          if (n_splits == 1) {
+            uint16_t* optr = out + (orow * H + hd * G + j_head) * D + h * 64 + c * 32;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv, __uint_as_float(o[i + 2 * e + 1]) * inv);
+                w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(optr + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else {
+            float* optr = part_o + slot * D + h * 64 + c * 32;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(optr + i) = make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
+                                                                 __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+          }
+        }
+      }
+      if (row_valid && h == 0) {
+        if (n_splits == 1) { if (lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = lse; }
+        else part_lse[slot] = lse;
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, tile, hd);
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // Explicit lists (the paper's controlled configurations): per target the index of the last context entry
 // at or before its position (-1: none), per context entry the row of the fresh K/V that replaces it (-1:
 // cached).  rt.tile_cu = prefix of the host bounds on the target counts, rt.bound_b = bounds on the context.
@@ -970,7 +1359,7 @@ __global__ void combine_splits_kernel(const float* __restrict__ part_o, const fl
 }
 
 static int g_forced_splits = 0;      // 0: chosen from the launch size; > 0: forced (test hook)
-static int g_sm_pairs = 0;           // 1: head_dim 128 runs on the SM-pair kernel (opt-in, test hook)
+static int g_variant = 0;            // head_dim 128 only (test hook): 0 two tiles per CTA, 1 SM pairs, 2 one tile with split keys
 
 // ---- host side ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1012,8 +1401,9 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   const int tile_targets = kBM / G;
   const int B = shape->n_req;
   // opt-in: head_dim 128 on SM pairs (a cluster of two CTAs = four query tiles); otherwise single CTAs
-  const bool use_pair = (D == 128) && g_sm_pairs;
-  const int tiles_per_unit = use_pair ? 4 : 2;
+  const bool use_pair = (D == 128) && g_variant == 1;
+  const bool use_split = (D == 128) && g_variant == 2;
+  const int tiles_per_unit = use_pair ? 4 : (use_split ? 1 : 2);
   for (int b = 0; b < B; ++b)     // tile_cu counts the launch units per request: tile PAIRS, or clusters of two pairs
     plan.rt.tile_cu[b + 1] = plan.rt.tile_cu[b] + (plan.rt.bound_a[b] + tiles_per_unit * tile_targets - 1) / (tiles_per_unit * tile_targets);
   const long long grid = (long long)plan.rt.tile_cu[B] * Hkv * (use_pair ? 2 : 1);
@@ -1058,12 +1448,17 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
   if (!attr_done[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_pair_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic) != cudaSuccess)
+        cudaFuncSetAttribute(attention_pair_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_split_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SplitSmem::kDynamic) != cudaSuccess)
       return RELAXKV_ERR_CUDA;
     attr_done[dev] = true;
   }
   if (use_pair) {
     attention_pair_sm100_kernel<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, PairSmem::kDynamic, stream>>>(
+        tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
+        u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
+  } else if (use_split) {
+    attention_split_sm100_kernel<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, SplitSmem::kDynamic, stream>>>(
         tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
         u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
   } else {
@@ -1106,8 +1501,9 @@ extern "C" relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits) {
   return RELAXKV_OK;
 }
 
-extern "C" relaxkv_status relaxkv_debug_set_attention_sm_pairs(int32_t on) {
-  g_sm_pairs = on ? 1 : 0;
+extern "C" relaxkv_status relaxkv_debug_set_attention_variant(int32_t variant) {
+  if (variant < 0 || variant > 2) return RELAXKV_ERR_INVALID_ARG;
+  g_variant = variant;
   return RELAXKV_OK;
 }
 

@@ -269,14 +269,16 @@ def test_context_split_matches_oracle(case, n_splits):
         B().relaxkv_debug_set_attention_splits(0)
 
 
+@pytest.mark.parametrize("variant", [1, 2], ids=["sm_pairs", "split_keys"])
 @pytest.mark.parametrize("n_splits", [0, 3])
-def test_sm_pair_kernel_matches_oracle(case, n_splits):
-    """The opt-in SM-pair variant (clusters of two blocks, one MMA instruction stream for both SMs, half of every
-    K/V tile per block) against the oracle, both context modes, with and without a forced context split; an odd
-    number of tile pairs leaves the last cluster's second block without targets."""
+def test_other_attention_kernels_match_oracle(case, n_splits, variant):
+    """The opt-in kernel variants for head_dim 128 - SM pairs (clusters of two blocks, one MMA instruction stream for
+    both SMs, half of every K/V tile per block; an odd number of tile pairs leaves the last cluster's second block
+    without targets) and one tile per block with S/P double-buffered and the keys split between the softmax
+    warpgroups - against the oracle, both context modes, with and without a forced context split."""
     s = case.make_session()
     s.build_active_sets(case.anchors_tensor())
-    B().relaxkv_debug_set_attention_sm_pairs(True)
+    B().relaxkv_debug_set_attention_variant(variant)
     B().relaxkv_debug_set_attention_splits(n_splits)
     try:
         for l in range(case.w.n_layers):
@@ -285,7 +287,7 @@ def test_sm_pair_kernel_matches_oracle(case, n_splits):
                 check_attention(case, l, out, lse, full_prefix)
     finally:
         B().relaxkv_debug_set_attention_splits(0)
-        B().relaxkv_debug_set_attention_sm_pairs(False)
+        B().relaxkv_debug_set_attention_variant(0)
 
 
 def test_attention_orders_agree_and_is_deterministic(case):
