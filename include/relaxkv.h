@@ -382,6 +382,13 @@ relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits);
 relaxkv_status relaxkv_debug_set_attention_variant(int32_t variant);
 
 /*
+ * Test utility (the paper has no counterpart).  relaxkv_linear / relaxkv_linear_swiglu run on SM pairs (clusters of
+ * two thread blocks, 256 x 256 tiles, one MMA instruction stream for both tensor cores); on != 0 makes every later
+ * call of this process use the single-block kernel (128 x 256 tiles), 0 restores the default.  Same results.
+ */
+relaxkv_status relaxkv_debug_set_gemm_single_cta(int32_t on);
+
+/*
  * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on
  * a barrier nothing will ever complete.  The wait gives up after its limit (0.4 s), the kernel ends
  * normally and RELAXKV_ERR_TIMEOUT is recorded in the device status word - the same path a stuck

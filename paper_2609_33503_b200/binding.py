@@ -23,7 +23,7 @@ ENTRY_POINTS = (
     "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
-    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_debug_set_attention_splits", "relaxkv_debug_set_attention_variant",
+    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_debug_set_attention_splits", "relaxkv_debug_set_attention_variant", "relaxkv_debug_set_gemm_single_cta",
     "relaxkv_list_attention", "relaxkv_cache_attention",
     "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_swiglu", "relaxkv_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
@@ -338,6 +338,11 @@ def relaxkv_debug_set_attention_variant(variant: int) -> None:
     """Kernel of head_dim-128 attention calls: 0 two tiles per block (default), 1 SM pairs, 2 one tile with split keys.
     Test hook."""
     _check(lib().relaxkv_debug_set_attention_variant(ctypes.c_int32(int(variant))), "relaxkv_debug_set_attention_variant")
+
+
+def relaxkv_debug_set_gemm_single_cta(on: bool) -> None:
+    """Run the GEMM calls on the single-block kernel instead of SM pairs (the default).  Test hook."""
+    _check(lib().relaxkv_debug_set_gemm_single_cta(ctypes.c_int32(1 if on else 0)), "relaxkv_debug_set_gemm_single_cta")
 
 
 def relaxkv_debug_wait_timeout(stream=None) -> None:

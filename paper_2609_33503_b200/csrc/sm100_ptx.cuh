@@ -248,14 +248,18 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
+// One arrival on a barrier of another CTA of the cluster.  Default qualifiers (release at CTA scope): a cluster-scope
+// release on every arrival measured ~2x slower kernels (each arrival then waits for the thread's earlier writes to
+// become visible cluster-wide); the data handed over here lives in tensor memory or was written by TMA and is ordered
+// by tcgen05.fence / the mbarrier's own completion.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok;
@@ -299,6 +303,15 @@ __device__ __forceinline__ void mma2_ss_kloop(uint32_t d_tmem, uint32_t a_lo, ui
       RELAXKV_MMA2_SS_STEP(1024, 512, p1) RELAXKV_MMA2_SS_STEP(1026, 514, p1) RELAXKV_MMA2_SS_STEP(1028, 516, p1)
       RELAXKV_MMA2_SS_STEP(1030, 518, p1)
       "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem] for four K steps of 16 inside one 64-element swizzled K block (both K-major).
+__device__ __forceinline__ void mma2_ss_4steps(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                               uint32_t acc_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      RELAXKV_MMA2_SS_STEP(0, 0, p0) RELAXKV_MMA2_SS_STEP(2, 2, p1) RELAXKV_MMA2_SS_STEP(4, 4, p1) RELAXKV_MMA2_SS_STEP(6, 6, p1)
+      "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc_first) : "memory");
 }
 #define RELAXKV_MMA2_TS_STEP(AOFF, BOFF, PRED)                                               \
   "add.u32 ta, %1, " #AOFF ";\n\tadd.u32 tb, %2, " #BOFF ";\n\t"                                  \

@@ -35,8 +35,18 @@ def close(got: torch.Tensor, ref: np.ndarray, abs_floor: float):
 
 
 @pytest.mark.parametrize("M,N,K,res", [(300, 512, 320, False), (129, 264, 72, True), (1000, 1024, 2048, True), (1, 8, 8, False),
-                                       (257, 1280, 640, False)])
-def test_linear(M, N, K, res):
+                                       (257, 1280, 640, False), (5000, 2304, 1024, True)])
+@pytest.mark.parametrize("single_cta", [False, True], ids=["sm_pairs", "single_cta"])
+def test_linear(M, N, K, res, single_cta):
+    """Both GEMM kernels: the default on SM pairs (256 x 256 tiles per cluster) and the single-block one."""
+    B().relaxkv_debug_set_gemm_single_cta(single_cta)
+    try:
+        _check_linear(M, N, K, res)
+    finally:
+        B().relaxkv_debug_set_gemm_single_cta(False)
+
+
+def _check_linear(M, N, K, res):
     x, w = rnd(M, K, seed=1), rnd(N, K, scale=K ** -0.5, seed=2)
     r = rnd(M, N, seed=3) if res else None
     y = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
