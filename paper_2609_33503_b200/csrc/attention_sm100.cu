@@ -798,13 +798,13 @@ attention_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __gr
         if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive_remote(ld_pfull);
+          if (cr == 0) mbar_arrive(bar_pfull + 8 * x); else mbar_arrive_remote(ld_pfull);
         }
       }
       z += (zs0 + zs1) + (zs2 + zs3);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive_remote(ld_pfull_hi);
+      if (cr == 0) mbar_arrive(bar_pfull_hi + 8 * x); else mbar_arrive_remote(ld_pfull_hi);
     }
     if (ok && my_n > 0) {
       ok = mbar_wait(bar_ofinal + 8 * x, 0, abort_flag);
