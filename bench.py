@@ -7,14 +7,18 @@ attention and the cache update.  Default workload: the Qwen3-14B-shaped 32K-cont
 at a 15 % anchor ratio (the configuration the headline metric is quoted on).
 
 Prints ONE JSON line.  `value` = algorithmic repair-attention TFLOP/s (4*D*H*edges) over the whole
-step time, inputs resident in HBM.  `--impl reference` times the fp64 CPU oracle on a bounded sample
-of the same workload instead.
+step time, inputs resident in HBM.  After the headline workload the default run also times the other
+benchmark configurations (the 16K single layer, the end points of the anchor-ratio sweep with their
+Full-Prefix Controls, the ragged batch of eight) with a few steps each and reports them under
+`other_configs`.  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same
+workload instead.  `--gpus N` without a launcher starts N local ranks itself (one GPU each).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -30,13 +34,15 @@ import torch
 from paper_2609_33503_b200 import inputs
 
 # Measured DRAM traffic of the attention kernel relative to its algorithmic bytes (Q rows in, O rows out, the
-# materialised context once): two ncu captures summarised in profiles/attention_sm100_qwen14b_32k_layer.md gave
-# 398 MB / 430 MB and 533 MB / 566 MB.  The capture rule forbids profiling the 20 GB stack with all sections;
-# both terms grow with the launch's rows and context, so a launch's traffic is this ratio x its algorithmic bytes.
+# materialised context once): ncu captures of a two-layer case gave 398 MB / 430 MB and 533 MB / 566 MB.  A capture
+# of the 20 GB stack with all sections is not allowed; both terms grow with the launch's rows and context, so a
+# launch's traffic is this ratio x its algorithmic bytes.
 ATTN_DRAM_TRAFFIC_OVER_ALGORITHMIC = 0.94
 
 METRIC = "repair_attention_tflops"
 UNIT = "TFLOP/s"
+N_SMS = 148
+EX2_PER_CLK_PER_SM = 16          # exponential unit: 4 lanes per scheduler, 4 schedulers per SM
 
 
 def load_peaks():
@@ -53,6 +59,8 @@ def make_workload(args) -> inputs.Workload:
         return inputs.qwen14b_32k(args.variant, args.ratio, args.layers or 40)
     if args.workload == "llama8b_16k":
         return inputs.llama8b_16k().replace(ratio=args.ratio)
+    if args.workload == "llama8b_8k":
+        return inputs.llama8b_stack(8192, args.layers or 32).replace(ratio=args.ratio)
     if args.workload == "tiny":
         return inputs.tiny().replace(ratio=args.ratio)
     if args.workload == "ragged8":
@@ -75,6 +83,22 @@ def whole_job_value(flops_per_rank: float, world: int, ms_per_step: float) -> fl
     return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
 
 
+def free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def launch_ranks(n: int, argv) -> int:
+    """Starts n local ranks of this script under torch.distributed.run (one process per GPU, rendezvous on
+    127.0.0.1) and returns the launcher's exit code.  Rank 0 prints the JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -93,6 +117,7 @@ class ClockSampler:
             self.t.start()
         except Exception:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
@@ -125,12 +150,14 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 
 class GpuJob:
+    """Device-resident inputs of one workload.  The per-layer caches do not depend on the anchor ratio;
+    `prepare(ratio)` runs one untimed selection pass and builds the "freshly recomputed" rows of the active
+    targets for that ratio."""
+
     def __init__(self, w: inputs.Workload, device):
         from paper_2609_33503_b200 import binding as B
-        from paper_2609_33503_b200.pipeline import RepairSession
         self.B, self.w, self.device = B, w, device
         nb, L = w.n_req, w.n_layers
-        self.k = [B.relaxkv_anchor_count(t, w.ratio) for t in w.ctx_lens]
         self.ctx_cu = np.concatenate([[0], np.cumsum(w.ctx_lens)]).astype(np.int64)
         offs = [int(x) for x in self.ctx_cu[:-1]]
         self.q_layers, self.k_naive, self.k_cache, self.v_cache = [], [], [], []
@@ -143,7 +170,17 @@ class GpuJob:
             self.v_cache.append(torch.cat(vs).contiguous())
         self.naive_views = [B.CacheView(k, None, offs) for k in self.k_naive]
         self.views = [B.CacheView(k, v, offs) for k, v in zip(self.k_cache, self.v_cache)]
-        self.s = RepairSession(w.n_q_heads, w.n_kv_heads, w.head_dim, w.ctx_lens, w.q_lens, L, self.k, device=device)
+        self.launches_per_step = 0
+        self.prepare(w.ratio)
+
+    def prepare(self, ratio: float, want_norm: bool = False):
+        from paper_2609_33503_b200.pipeline import RepairSession
+        B, device = self.B, self.device
+        self.w = w = self.w.replace(ratio=ratio)
+        nb, L = w.n_req, w.n_layers
+        self.k = [B.relaxkv_anchor_count(t, w.ratio) for t in w.ctx_lens]
+        self.s = RepairSession(w.n_q_heads, w.n_kv_heads, w.head_dim, w.ctx_lens, w.q_lens, L, self.k, device=device,
+                               want_norm=want_norm)
         # untimed set-up pass: the sets decide which rows are "freshly recomputed"
         self.s.score_select(self.q_layers, self.naive_views)
         self.s.build_active_sets()
@@ -165,13 +202,12 @@ class GpuJob:
             self.fresh.append([torch.cat(qs).contiguous(), torch.cat(ks).contiguous(), torch.cat(vs).contiguous()])
             self.edges.append(e); self.edges_full.append(ef)
         self.outs = [torch.empty_like(f[0]) for f in self.fresh]
-        self.launches_per_step = 0
 
     # one pass of the whole hot path; `ev` collects (phase, start event, end event)
     def step(self, ev=None, mode=None):
         B, s, w = self.B, self.s, self.w
         mode = B.CTX_UNION if mode is None else mode
-        nb, L = w.n_req, w.n_layers
+        L = w.n_layers
 
         def rec(name, fn):
             if ev is None:
@@ -212,10 +248,167 @@ class GpuJob:
             total = sum(a.elapsed_time(b_) for a, b_ in evs)
         return total
 
+    def time_attention_stream(self, mode, reps: int):
+        """ms per pass over the layers' attention calls when `reps` passes are queued back to back with no host
+        synchronisation in between: what a caller that keeps the stream fed sees (for short calls the per-step figure
+        also contains the host's launch work, because every step starts after a host sync)."""
+        s = self.s
+        n_u, n_r = s.counts()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for timed in (False, True):
+            if timed:
+                a.record()
+            for _ in range(reps):
+                for l in range(self.w.n_layers):
+                    f = self.fresh[l]
+                    s.attention(l, self.views[l], f[0], f[1], f[2], self.outs[l], n_r[l], n_u, mode=mode)
+            if timed:
+                b_.record()
+            torch.cuda.synchronize()
+        return a.elapsed_time(b_) / reps
+
     def flops(self, full_prefix=False):
         w = self.w
         e = sum(self.edges_full if full_prefix else self.edges)
         return 4.0 * w.head_dim * w.n_q_heads * e
+
+
+def check_status(B):
+    st, detail = B.relaxkv_read_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {B.status_string(st)} {detail}")
+
+
+def measure(job: GpuJob, full_prefix: bool, steps: int, warmup: int, peaks, device_index: int, world: int = 1,
+            barrier=None, sample_clocks: bool = True):
+    """Warm-up, then `steps` timed steps of the whole path; returns the figures of one benchmark line."""
+    B, w = job.B, job.w
+    mode = B.CTX_FULL_PREFIX if full_prefix else B.CTX_UNION
+    for _ in range(warmup):
+        job.step(mode=mode)
+    torch.cuda.synchronize()
+    check_status(B)
+    sampler = None
+    if sample_clocks:
+        sampler = ClockSampler(device_index).start()
+        time.sleep(0.3)
+    if barrier:
+        barrier()
+    ev = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        job.step(ev, mode=mode)
+    t1.record()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    elapsed_ms = t0.elapsed_time(t1)
+    clocks = sampler.stop() if sampler else None
+    elapsed_ms = max_over_ranks(elapsed_ms, job.device, world)
+    check_status(B)
+    phase_ms = {}
+    for name, a, b_ in ev:
+        phase_ms[name] = phase_ms.get(name, 0.0) + a.elapsed_time(b_)
+    phase_ms = {k: v / steps for k, v in phase_ms.items()}
+    ms_per_step = elapsed_ms / steps
+    gather_ms = job.time_gather(mode)
+    L = w.n_layers
+    flops = job.flops(full_prefix)
+    kv_row = w.n_kv_heads * w.head_dim * 2
+    sum_t = int(job.ctx_cu[-1])
+    ctx_rows = sum(job.n_u) if not full_prefix else sum_t
+    scatter_bytes = sum(2 * 2 * sum(nr) * kv_row for nr in job.n_r)           # K and V, read + write
+    gather_bytes = L * 2 * 2 * ctx_rows * kv_row                               # K and V, read + write
+    attn_tflops = flops / (phase_ms["attention"] * 1e-3) / 1e12
+    mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
+    # scoring: two passes of Q K^T over every cached key, one exponential per logit and pass
+    hq_t = sum(q * t for q, t in zip(w.q_lens, w.ctx_lens)) * w.n_q_heads
+    score_flops = L * 2 * 2.0 * hq_t * w.head_dim
+    score_ex2 = L * 2.0 * hq_t
+    t_sel = phase_ms["score_select"] * 1e-3
+    scoring = {"us": round(t_sel * 1e6, 1), "tflops": round(score_flops / t_sel / 1e12, 1),
+               "frac_of_sustained_bf16_peak": round(score_flops / t_sel / 1e12 / peaks["bf16_tflops_sustained"], 4),
+               "ex2_per_s": float(f"{score_ex2 / t_sel:.4g}"), "binder": "mufu",
+               "k_bytes_once_gbs": round(L * sum_t * kv_row / t_sel / 1e9, 1),
+               "note": "K bytes once / time is not the binder: at G*Q query rows per KV head every key byte feeds "
+                       "thousands of flops and several exponentials; the exponential unit binds, then the tensor pipe"}
+    if mhz:
+        scoring["frac_of_ex2_ceiling"] = round(score_ex2 / t_sel / (EX2_PER_CLK_PER_SM * N_SMS * mhz * 1e6), 4)
+        scoring["ex2_ceiling"] = f"{EX2_PER_CLK_PER_SM} ex2/clk/SM x {N_SMS} SMs x {mhz:.0f} MHz (median sampled clock)"
+    out = {
+        "ms_per_step": round(ms_per_step, 3), "flops": flops,
+        "phases_us": {k: round(v * 1e3, 1) for k, v in phase_ms.items()},
+        "sets": {"ctx_ratio": round(sum(job.n_u) / sum_t, 4),
+                 "active_ratio": round(sum(sum(x) for x in job.n_r) / (L * sum_t), 4),
+                 "edges": int(sum(job.edges)), "edges_full_prefix": int(sum(job.edges_full))},
+        "attention_tflops": round(attn_tflops, 2),
+        "attention_frac_of_sustained_peak": round(attn_tflops / peaks["bf16_tflops_sustained"], 4),
+        "scatter_gbs": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9, 1),
+        "scatter_frac_hbm": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "gather_us": round(gather_ms * 1e3, 1),
+        "gather_gbs": round(gather_bytes / (gather_ms * 1e-3) / 1e9, 1),
+        "gather_frac_hbm": round(gather_bytes / (gather_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "scoring": scoring, "clocks": clocks,
+    }
+    if mhz:
+        # cycle-normalised: time x median sampled SM clock, so that power-cap clock drift between runs does not pass
+        # for a change of the kernel
+        cyc = phase_ms["attention"] * 1e-3 * mhz * 1e6
+        out["attention_cycles"] = {"gcycles_per_step": round(cyc / 1e9, 4),
+                                   "flop_per_clk_per_sm": round(flops / cyc / N_SMS, 1),
+                                   "how": "attention phase time x median sampled SM MHz"}
+    out["_gather_ms"], out["_phase_ms"], out["_ctx_rows"], out["_kv_row"] = gather_ms, phase_ms, ctx_rows, kv_row
+    return out
+
+
+def other_configs(args, peaks, device, main_job: GpuJob):
+    """The remaining benchmark configurations, a few steps each: the Llama-3.1-8B-shaped 16K layer, the end points
+    of the anchor-ratio sweep on the 32K stack (each with its Full-Prefix Control, same targets) and the ragged
+    batch of eight requests (8 layers).  Same measurement as the headline line."""
+    res = {}
+    steps, warm = 3, 3
+    idx = device.index or 0
+
+    def brief(m, job):
+        keys = ("ms_per_step", "phases_us", "sets", "attention_tflops", "attention_frac_of_sustained_peak", "gather_gbs",
+                "gather_frac_hbm", "scatter_gbs", "scatter_frac_hbm", "attention_cycles")
+        d = {k: m[k] for k in keys if k in m}
+        d["clock_mhz"] = m["clocks"]["sm_mhz"] if m.get("clocks") else None
+        d["value_tflops"] = round(m["flops"] / (m["ms_per_step"] * 1e-3) / 1e12, 2)
+        d["n_layers"] = job.w.n_layers
+        return d
+
+    # anchor-ratio sweep end points on the headline workload's caches
+    if main_job.w.name.startswith("qwen14b_32k"):
+        base_ratio = main_job.w.ratio
+        for r in (0.05, 0.30):
+            main_job.prepare(r)
+            key = f"qwen14b_32k_r{int(round(r * 100)):02d}"
+            mu = measure(main_job, False, steps, warm, peaks, idx)
+            mf = measure(main_job, True, steps, warm, peaks, idx)
+            res[key] = brief(mu, main_job)
+            res[key + "_full_prefix"] = brief(mf, main_job)
+            res[key]["attention_time_saved_vs_full_prefix"] = round(1.0 - mu["_phase_ms"]["attention"] / mf["_phase_ms"]["attention"], 4)
+        main_job.prepare(base_ratio)
+    # 16K single layer: a 100-microsecond call, so the per-step figure is dominated by the host's launch work
+    # between two syncs; the stream figure queues 20 passes back to back
+    job = GpuJob(inputs.llama8b_16k(), device)
+    m = measure(job, False, 10, warm, peaks, idx)
+    d = brief(m, job)
+    ms_stream = job.time_attention_stream(job.B.CTX_UNION, 20)
+    d["attention_stream_us"] = round(ms_stream * 1e3, 1)
+    d["attention_stream_tflops"] = round(job.flops() / (ms_stream * 1e-3) / 1e12, 1)
+    res["llama8b_16k"] = d
+    del job
+    torch.cuda.empty_cache()
+    # ragged batch of eight, all requests in one launch per call
+    job = GpuJob(inputs.ragged8(8), device)
+    m = measure(job, False, steps, warm, peaks, idx)
+    res["ragged8_8layers"] = brief(m, job)
+    del job
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_gpu(args):
@@ -231,16 +424,7 @@ def run_gpu(args):
         raise SystemExit("librelaxkv.so is missing: run `python __graft_entry__.py` first (no CPU fallback exists)")
     w = make_workload(args)
     peaks = load_peaks()
-    if args.attn_variant:
-        B.relaxkv_debug_set_attention_variant(args.attn_variant)
     job = GpuJob(w, device)
-    mode = B.CTX_FULL_PREFIX if args.full_prefix else B.CTX_UNION
-    for _ in range(args.warmup):
-        job.step(mode=mode)
-    torch.cuda.synchronize()
-    st, detail = B.relaxkv_read_device_status()
-    if st != 0:
-        raise SystemExit(f"device status {B.status_string(st)} {detail}")
 
     def barrier():
         if world > 1:
@@ -248,57 +432,37 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    barrier()
-    ev = []
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(args.steps):
-        job.step(ev, mode=mode)
-    t1.record()
-    barrier()
-    elapsed_ms = t0.elapsed_time(t1)
-    clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = max_over_ranks(elapsed_ms, device, world)
-    st, detail = B.relaxkv_read_device_status()
-    if st != 0:
-        raise SystemExit(f"device status {B.status_string(st)} {detail}")
-
-    phase_ms = {}
-    for name, a, b_ in ev:
-        phase_ms[name] = phase_ms.get(name, 0.0) + a.elapsed_time(b_)
-    phase_ms = {k: v / args.steps for k, v in phase_ms.items()}
-    ms_per_step = elapsed_ms / args.steps
-    flops = job.flops(args.full_prefix)
+    m = measure(job, args.full_prefix, args.steps, args.warmup, peaks, local, world, barrier, sample_clocks=(rank == 0))
+    mode = B.CTX_FULL_PREFIX if args.full_prefix else B.CTX_UNION
+    ms_per_step = m["ms_per_step"]
+    flops = m["flops"]
     value = whole_job_value(flops, world, ms_per_step)
-
-    # ---- the gather step on its own (it runs inside every attention call) -------------------------------
-    gather_ms = job.time_gather(mode)
 
     # ---- end-to-end arm: host buffers, copies inside the timed region --------------------------------
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(job, args, mode, world)
 
+    others = None
+    if rank == 0 and world == 1 and not args.no_others and args.workload == "qwen14b_32k" and not args.full_prefix:
+        others = other_configs(args, peaks, device, job)
+
     if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
         return
     L = w.n_layers
-    attn_tflops = flops / (phase_ms["attention"] * 1e-3) / 1e12
-    kv_row = w.n_kv_heads * w.head_dim * 2
-    scatter_bytes = sum(2 * 2 * sum(nr) * kv_row for nr in job.n_r)          # K and V, read + write
-    sum_t = int(job.ctx_cu[-1])
-    ctx_rows = sum(job.n_u) if not args.full_prefix else sum_t
-    gather_bytes = L * 2 * 2 * ctx_rows * kv_row                               # K and V, read + write
+    phase_ms, gather_ms = m["_phase_ms"], m["_gather_ms"]
     # launch-bound cases (gather time comparable to the whole call) have no meaningful difference
     attn_kernel_ms = phase_ms["attention"] - gather_ms if gather_ms < 0.5 * phase_ms["attention"] else None
-    alg_bytes = 2 * sum(sum(x) for x in job.n_r) / L * w.n_q_heads * w.head_dim * 2 + 2 * ctx_rows * kv_row
+    alg_bytes = 2 * sum(sum(x) for x in job.n_r) / L * w.n_q_heads * w.head_dim * 2 + 2 * m["_ctx_rows"] * m["_kv_row"]
     traffic = {"bytes_per_launch": round(ATTN_DRAM_TRAFFIC_OVER_ALGORITHMIC * alg_bytes),
                "algorithmic_bytes_per_launch": round(alg_bytes),
-               "how": "ncu dram read+write of captured launches on a smaller case = 0.94 x their algorithmic bytes; scaled"}
-    select_bytes = L * sum_t * w.n_kv_heads * w.head_dim * 2                  # each layer's K read once
+               "how": "ncu dram read+write of captured launches on a smaller case = 0.94 x their algorithmic bytes; scaled "
+                      "(not a measurement of this run)"}
+    attn_tflops = m["attention_tflops"]
     out = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
@@ -309,27 +473,28 @@ def run_gpu(args):
                    "l2": "inputs larger than L2 (per-layer K/V and Q/O buffers total several GB)",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "layer_stack_us": round(ms_per_step * 1e3, 1),
-        "phases_us": {k: round(v * 1e3, 1) for k, v in phase_ms.items()},
-        "sets": {"ctx_ratio": round(sum(job.n_u) / sum_t, 4),
-                 "active_ratio": round(sum(sum(x) for x in job.n_r) / (L * sum_t), 4),
-                 "edges": int(sum(job.edges)), "edges_full_prefix": int(sum(job.edges_full))},
-        "scatter_gbs": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9, 1),
-        "scatter_frac_hbm": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
-        "select_gbs": round(select_bytes / (phase_ms["score_select"] * 1e-3) / 1e9, 1),
-        "gather_us": round(gather_ms * 1e3, 1),
-        "gather_gbs": round(gather_bytes / (gather_ms * 1e-3) / 1e9, 1),
-        "gather_frac_hbm": round(gather_bytes / (gather_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
-        "roofline": {"bound": "tensor", "achieved": round(attn_tflops, 2), "peak": peaks["bf16_tflops_sustained"],
+        "phases_us": m["phases_us"], "sets": m["sets"],
+        "scatter_gbs": m["scatter_gbs"], "scatter_frac_hbm": m["scatter_frac_hbm"],
+        "gather_us": m["gather_us"], "gather_gbs": m["gather_gbs"], "gather_frac_hbm": m["gather_frac_hbm"],
+        "scoring": m["scoring"],
+        "roofline": {"bound": "tensor", "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": round(attn_tflops / peaks["bf16_tflops_sustained"], 4),
                      "frac_of_burst_peak": round(attn_tflops / peaks["bf16_tflops"], 4),
                      "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
                      "kernel": "attention_sm100_kernel (timed per call, which includes its gather launch)",
-                     "achieved_without_gather": round(flops / (attn_kernel_ms * 1e-3) / 1e12, 2) if attn_kernel_ms else None},
-        "clocks": clocks, "gpu_launches": job.launches_per_step * args.steps, "e2e": e2e,
+                     "achieved_without_gather": round(flops / (attn_kernel_ms * 1e-3) / 1e12, 2) if attn_kernel_ms else None,
+                     "cycles": m.get("attention_cycles")},
+        "clocks": m["clocks"], "gpu_launches": job.launches_per_step * args.steps, "e2e": e2e,
     }
+    if others is not None:
+        out["other_configs"] = others
     if not args.no_cpu and world == 1:
-        out["cpu_baseline"] = cpu_baseline(w, args, job)
+        out["cpu_baseline"] = cpu_baseline(w, args, sum(job.edges_full if args.full_prefix else job.edges))
     print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
 
 
 def run_e2e(job, args, mode, world):
@@ -367,6 +532,164 @@ def run_e2e(job, args, mode, world):
             "steps": n, "how": "pinned host buffers, 3 streams (copy-in | kernels | copy-out), 3 layers in flight"}
 
 
+# --------------------------------------------------------------------------------------------------
+# controlled configurations (explicit target / context lists)
+# --------------------------------------------------------------------------------------------------
+
+LIST_CONFIGS = ("relaxkv_g", "global_sparse", "layerwise_sparse", "target_sweep", "target_union")
+
+
+class ListJob:
+    """One of the paper's controlled configurations on the explicit-list entry points.  Per step: scoring and top-k
+    for every layer, the repair schedule, the across-layer mean score and the extra top-k the configuration needs,
+    then per layer relaxkv_list_attention and relaxkv_scatter_kv_lists.
+      relaxkv_g         targets: one global list P = top-m of g (m = the mean of |R_l| over the layers, so the layer-token
+                        states match the method's), context U
+      target_sweep      targets: P = top-min(floor(r_g T_c), |U|) of g, context U
+      target_union      targets: P = top-|U| of g (the count of U, not U itself), context U
+      global_sparse     targets R_l, context = top-|U| of g, shared by the layers
+      layerwise_sparse  targets R_l, context U_l = top-|U| of layer l's own score
+    g_i = mean over layers of the MinMax-normalised scores."""
+
+    def __init__(self, job: GpuJob, config: str, rg: float):
+        self.job, self.config, self.rg = job, config, rg
+        B, w, dev = job.B, job.w, job.device
+        self.B = B
+        nb, L = w.n_req, w.n_layers
+        job.prepare(w.ratio, want_norm=True)
+        s = job.s
+        self.n_u, self.n_r = s.counts()
+        sum_t = int(job.ctx_cu[-1])
+        self.g = torch.empty(sum_t, dtype=torch.float32, device=dev)
+        self.global_targets = config in ("relaxkv_g", "target_sweep", "target_union")
+        if config == "relaxkv_g":
+            self.m = [max(1, int(round(sum(self.n_r[l][b] for l in range(L)) / L))) for b in range(nb)]
+        elif config == "target_sweep":
+            self.m = [max(1, min(int(np.floor(rg * t)), u)) for t, u in zip(w.ctx_lens, self.n_u)]
+        else:
+            self.m = list(self.n_u)                       # target_union and the two context variants: |U_b| entries
+        self.m_cu = np.concatenate([[0], np.cumsum(self.m)]).astype(np.int32)
+        self.sel = torch.empty((L if config == "layerwise_sparse" else 1), int(self.m_cu[-1]), dtype=torch.int32, device=dev)
+        self.sel_cu = torch.from_numpy(self.m_cu).to(dev)
+        self.u_cu_host = np.concatenate([[0], np.cumsum(self.n_u)]).astype(np.int32)
+        # targets R_l as positions (context variants): [L] tensors + rebased offsets, refreshed every step
+        self.rpos = [torch.empty(max(1, sum(self.n_r[l])), dtype=torch.int32, device=dev) for l in range(L)]
+        r_cu = np.zeros((L, nb + 1), dtype=np.int32)
+        for l in range(L):
+            r_cu[l, 1:] = np.cumsum(self.n_r[l])
+        self.r_cu_rebased = torch.from_numpy(r_cu).to(dev)
+        self._select()                                    # untimed: the lists decide which rows are "fresh"
+        torch.cuda.synchronize()
+        sel = self.sel.cpu().numpy()
+        u_pos = s.u_pos.cpu().numpy()
+        self.fresh, self.outs, self.edges = [], [], 0
+        for l in range(L):
+            qs, ks, vs = [], [], []
+            rpos_l = self.rpos[l].cpu().numpy()
+            for b in range(nb):
+                lo, hi = int(job.ctx_cu[b]), int(job.ctx_cu[b + 1])
+                if self.global_targets:
+                    tgt = sel[0, self.m_cu[b]:self.m_cu[b + 1]].astype(np.int64)
+                    ctx = u_pos[self.u_cu_host[b]:self.u_cu_host[b + 1]].astype(np.int64)
+                else:
+                    tgt = rpos_l[r_cu[l, b]:r_cu[l, b + 1]].astype(np.int64)
+                    row = l if config == "layerwise_sparse" else 0
+                    ctx = sel[row, self.m_cu[b]:self.m_cu[b + 1]].astype(np.int64)
+                self.edges += int(np.searchsorted(ctx, tgt, side="right").sum())
+                q, k, v = inputs.fresh_qkv(w, l, b, job.k_naive[l][lo:hi], job.v_cache[l][lo:hi], torch.from_numpy(tgt))
+                qs.append(q); ks.append(k); vs.append(v)
+            self.fresh.append([torch.cat(qs).contiguous(), torch.cat(ks).contiguous(), torch.cat(vs).contiguous()])
+            self.outs.append(torch.empty_like(self.fresh[-1][0]))
+        self.launches_per_step = 0
+
+    def _select(self):
+        """The list-building kernels of one step (after the schedule is known)."""
+        B, s, w = self.B, self.job.s, self.job.w
+        L = w.n_layers
+        if self.config == "layerwise_sparse":
+            B.relaxkv_select_topk(s.shape, L, self.m, s.raw, self.sel)
+        else:
+            B.relaxkv_mean_scores(s.shape, L, s.norm, self.g)
+            B.relaxkv_select_topk(s.shape, 1, self.m, self.g, self.sel)
+        if not self.global_targets:
+            for l in range(L):
+                B.relaxkv_target_positions(s.shape, s.u_pos, s.u_cu, s.r_rank, s.r_cu_layer(l), self.n_r[l], self.rpos[l])
+
+    def step(self, ev=None):
+        B, job, s, w = self.B, self.job, self.job.s, self.job.w
+        L = w.n_layers
+
+        def rec(name, fn):
+            if ev is None:
+                fn(); return
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b_.record(); ev.append((name, a, b_))
+
+        rec("score_select", lambda: s.score_select(job.q_layers, job.naive_views))
+        rec("build_sets", lambda: s.build_active_sets())
+        s.counts()
+        rec("lists", self._select)
+        for l in range(L):
+            f = self.fresh[l]
+            if self.global_targets:
+                ctx_pos, ctx_cu, tgt_pos, tgt_cu, mt = s.u_pos, s.u_cu, self.sel[0], self.sel_cu, self.m
+            else:
+                row = l if self.config == "layerwise_sparse" else 0
+                ctx_pos, ctx_cu, tgt_pos, tgt_cu, mt = self.sel[row], self.sel_cu, self.rpos[l], self.r_cu_rebased[l], self.n_r[l]
+            mc = self.n_u if self.global_targets else self.m
+            rec("attention", lambda: B.relaxkv_list_attention(s.shape, job.views[l], f[0], f[1], f[2], ctx_pos, ctx_cu, tgt_pos,
+                                                              tgt_cu, mt, mc, self.outs[l], s.workspace))
+            rec("scatter", lambda: B.relaxkv_scatter_kv_lists(s.shape, job.views[l], f[1], f[2], tgt_pos, tgt_cu, mt))
+        n_lists = (1 if self.config == "layerwise_sparse" else 2) + (0 if self.global_targets else L)
+        self.launches_per_step = 4 * ((L + 47) // 48) + 1 + 5 + n_lists + 4 * L      # per layer: maps, gather, attention, scatter
+
+
+def run_list_config(args):
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    from paper_2609_33503_b200 import binding as B
+    w = make_workload(args)
+    peaks = load_peaks()
+    job = GpuJob(w, device)
+    lj = ListJob(job, args.config, args.rg)
+    for _ in range(args.warmup):
+        lj.step()
+    torch.cuda.synchronize()
+    check_status(B)
+    sampler = ClockSampler(0).start()
+    time.sleep(0.3)
+    ev = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        lj.step(ev)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    check_status(B)
+    ms = t0.elapsed_time(t1) / args.steps
+    phase = {}
+    for name, a, b_ in ev:
+        phase[name] = phase.get(name, 0.0) + a.elapsed_time(b_) / args.steps
+    flops = 4.0 * w.head_dim * w.n_q_heads * lj.edges
+    sum_t = int(job.ctx_cu[-1])
+    n_tgt = sum(f[0].shape[0] for f in lj.fresh)
+    out = {"metric": METRIC, "value": round(flops / (ms * 1e-3) / 1e12, 3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": round(ms, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": w.name, "configuration": args.config, "n_layers": w.n_layers, "anchor_ratio": w.ratio,
+                      "global_target_ratio": args.rg if args.config == "target_sweep" else None,
+                      "ctx_lens": list(w.ctx_lens), "l2": "inputs larger than L2"},
+           "phases_us": {k: round(v * 1e3, 1) for k, v in phase.items()},
+           "sets": {"ctx_ratio": round(sum(lj.n_u if lj.global_targets else lj.m) / sum_t, 4),
+                    "active_ratio": round(n_tgt / (w.n_layers * sum_t), 4), "edges": int(lj.edges),
+                    "edges_relaxkv": int(sum(job.edges)), "edges_full_prefix": int(sum(job.edges_full))},
+           "attention_tflops": round(flops / (phase["attention"] * 1e-3) / 1e12, 2),
+           "attention_frac_of_sustained_peak": round(flops / (phase["attention"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
+           "clocks": clocks, "gpu_launches": lj.launches_per_step * args.steps}
+    print(json.dumps(out))
+
+
 def run_query_attention(args):
     """Attention of the user query over the (repaired) context cache with the same kernel, through
     relaxkv_list_attention: the query's prefill rows (the workload's Q rows, every context position visible)
@@ -398,23 +721,22 @@ def run_query_attention(args):
         ws = ws[off:off + nbytes]
         res = {}
         for label, forced in (("unsplit_us", 1), ("us", 0)):
-            B.relaxkv_debug_set_attention_splits(forced)
-            try:
-                def call():
-                    B.relaxkv_list_attention(shape, view, q, None, None, ctx_pos, ctx_cu, tgt_pos, tgt_cu, [Q], [T], o, ws)
-                for _ in range(max(3, args.warmup)):
-                    call()
-                torch.cuda.synchronize()
-                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                n = max(10, args.steps)
-                a.record()
-                for _ in range(n):
-                    call()
-                b_.record()
-                torch.cuda.synchronize()
-                res[label] = round(a.elapsed_time(b_) / n * 1e3, 1)
-            finally:
-                B.relaxkv_debug_set_attention_splits(0)
+            shape_f = B.Shape(H, Hkv, D, [T], [Q], attention_ctx_splits=forced)
+
+            def call():
+                B.relaxkv_list_attention(shape_f, view, q, None, None, ctx_pos, ctx_cu, tgt_pos, tgt_cu, [Q], [T], o, ws)
+            for _ in range(max(3, args.warmup)):
+                call()
+            torch.cuda.synchronize()
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(10, args.steps)
+            a.record()
+            for _ in range(n):
+                call()
+            b_.record()
+            torch.cuda.synchronize()
+            res[label] = round(a.elapsed_time(b_) / n * 1e3, 1)
+
         # cache-only entry point: no gather, K and V move once
         def call_cache():
             B.relaxkv_cache_attention(shape, view, q, tgt_pos, tgt_cu, [Q], o, ws)
@@ -433,9 +755,7 @@ def run_query_attention(args):
         res["kv_bytes"] = 2 * T * Hkv * D * 2
         res["cache_only_kv_gbs"] = round(res["kv_bytes"] / (res["cache_only_us"] * 1e-6) / 1e9, 1)
         out[name] = res
-    st, detail = B.relaxkv_read_device_status()
-    if st != 0:
-        raise SystemExit(f"device status {B.status_string(st)} {detail}")
+    check_status(B)
     out["value"] = out["prefill"]["cache_only_us"]
     print(json.dumps(out))
 
@@ -486,9 +806,7 @@ def run_dense(args):
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
-    st, detail = B.relaxkv_read_device_status()
-    if st != 0:
-        raise SystemExit(f"device status {B.status_string(st)} {detail}")
+    check_status(B)
     sampler = ClockSampler(0)
     sampler.start(); time.sleep(0.3)
     ev = []
@@ -559,33 +877,38 @@ def oracle_sample(w: inputs.Workload, n_rows: int, layer: int = 0, score_frac: f
     orc.repair_attention(kb, vb, qnb, knb, vnb, sets.u_pos, sets.ranks(0), scale, rows=rows)
     t_attn = time.perf_counter() - t0
     e_sample = int(sets.ranks(0)[rows].astype(np.int64).sum() + len(rows))
+    # edges per layer of request 0 under the sample's own schedule (mean over its 8 pseudo-layers)
+    e_layer = float(np.mean([orc.edges(sets.ranks(l)) for l in range(8)]))
     return {"t_score_layer_req": t_score, "t_attn_sample": t_attn, "edges_sample": e_sample, "rows": int(len(rows)),
-            "score_keys": n_keys, "threads": orc.n_threads()}
+            "score_keys": n_keys, "threads": orc.n_threads(), "edges_layer_req0": e_layer}
 
 
-def cpu_baseline(w, args, job=None):
-    n_rows = args.cpu_rows
-    smp = oracle_sample(w, n_rows)
-    if job is not None:
-        edges = sum(job.edges_full if args.full_prefix else job.edges)
-    else:
-        edges = None
-    out = {"kind": "oracle", "cores": smp["threads"], "unit": UNIT,
-           "sample": (f"fp64 oracle, request 0 / layer 0: scoring of the first {smp['score_keys']} context keys (scaled to "
-                      f"{smp['t_score_layer_req']:.2f} s per layer) + repair attention of {smp['rows']} target rows spread "
-                      f"over the staircase, all heads ({smp['edges_sample']} edges, {smp['t_attn_sample']:.2f} s)")}
+def oracle_step_rate(w: inputs.Workload, smp, edges_total=None):
+    """Whole-step oracle throughput from one sample - the ONE formula both arms use: scoring time scales with
+    layers x (query tokens x context tokens), attention time with edges.
+    edges_total: the workload's edges where they are known (the CUDA arm has run the path); otherwise the edges of
+    the sample's own schedule, scaled to every request by (T_b / T_0)^2 and to every layer."""
+    tok_scale = sum(t * q for t, q in zip(w.ctx_lens, w.q_lens)) / (w.ctx_lens[0] * w.q_lens[0])
+    if edges_total is None:
+        edges_total = w.n_layers * smp["edges_layer_req0"] * sum((t / w.ctx_lens[0]) ** 2 for t in w.ctx_lens)
+    t_step = smp["t_score_layer_req"] * w.n_layers * tok_scale + smp["t_attn_sample"] * edges_total / smp["edges_sample"]
+    return 4.0 * w.head_dim * w.n_q_heads * edges_total / t_step / 1e12, t_step
+
+
+def sample_text(smp):
+    return (f"fp64 oracle, request 0 / one layer: scoring of the first {smp['score_keys']} context keys (scaled to "
+            f"{smp['t_score_layer_req']:.2f} s per layer) + repair attention of {smp['rows']} target rows spread "
+            f"over the staircase, all heads ({smp['edges_sample']} edges, {smp['t_attn_sample']:.2f} s); whole-step time "
+            f"extrapolated in proportion to layers x tokens (scoring) and edges (attention)")
+
+
+def cpu_baseline(w, args, edges_total=None):
+    smp = oracle_sample(w, args.cpu_rows)
+    v, t_step = oracle_step_rate(w, smp, edges_total)
     flops_sample = 4.0 * w.head_dim * w.n_q_heads * smp["edges_sample"]
-    out["attention_only_value"] = round(flops_sample / smp["t_attn_sample"] / 1e12, 6)
-    if edges is not None:
-        # whole-step estimate: scoring scales with layers x context tokens, attention with edges
-        tok_scale = sum(t * q for t, q in zip(w.ctx_lens, w.q_lens)) / (w.ctx_lens[0] * w.q_lens[0])
-        t_step = smp["t_score_layer_req"] * w.n_layers * tok_scale + smp["t_attn_sample"] * edges / smp["edges_sample"]
-        out["value"] = round(4.0 * w.head_dim * w.n_q_heads * edges / t_step / 1e12, 6)
-        out["extrapolated_step_seconds"] = round(t_step, 1)
-        out["sample"] += "; whole-step time extrapolated in proportion to layers and edges"
-    else:
-        out["value"] = out["attention_only_value"]
-    return out
+    return {"kind": "oracle", "cores": smp["threads"], "unit": UNIT, "sample": sample_text(smp), "value": round(v, 6),
+            "attention_only_value": round(flops_sample / smp["t_attn_sample"] / 1e12, 6),
+            "extrapolated_step_seconds": round(t_step, 1)}
 
 
 def run_reference(args):
@@ -599,35 +922,42 @@ def run_reference(args):
     vals = []
     for i in range(args.steps):
         smp = oracle_sample(w, args.cpu_rows, layer=i % w.n_layers)
-        # edges of the full workload are unknown without running the path: rate = sampled flops / sampled time,
-        # with the scoring share charged per edge at the workload's nominal ratio of scoring to attention work
-        flops_sample = 4.0 * w.head_dim * w.n_q_heads * smp["edges_sample"]
-        vals.append(flops_sample / (smp["t_attn_sample"] + smp["t_score_layer_req"] * smp["edges_sample"] /
-                                    max(1, nominal_edges_per_layer(w))) / 1e12)
+        vals.append(oracle_step_rate(w, smp)[0])
     ms = (time.perf_counter() - t0) * 1e3 / args.steps
     v = float(np.mean(vals))
-    sample = (f"fp64 oracle on host cores: per step, scoring of a quarter of one layer's context keys (scaled to the layer) and "
-              f"repair attention of {args.cpu_rows} target rows spread over the staircase (all heads); rate = sampled "
-              f"attention flops / (attention time + scoring time charged in proportion to edges)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(v, 6), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", 1)),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "n_layers": w.n_layers, "anchor_ratio": w.ratio, "ctx_lens": list(w.ctx_lens)},
-        "cpu_baseline": {"kind": "oracle", "cores": smp["threads"], "sample": sample, "value": round(v, 6), "unit": UNIT},
+        "config": {"workload": w.name, "n_layers": w.n_layers, "heads": f"{w.n_q_heads}/{w.n_kv_heads}", "head_dim": w.head_dim,
+                   "ctx_lens": list(w.ctx_lens), "q_lens": list(w.q_lens), "anchor_ratio": w.ratio,
+                   "context": "full_prefix" if args.full_prefix else "union"},
+        "cpu_baseline": {"kind": "oracle", "cores": smp["threads"], "sample": sample_text(smp), "value": round(v, 6), "unit": UNIT},
         "e2e": {"value": round(v, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def nominal_edges_per_layer(w):
-    """Edges of one layer if this layer's anchors alone formed U = R (a lower bound used only to
-    apportion the oracle's scoring time in the reference arm)."""
-    from oracle import relaxkv_oracle as orc
-    e = 0
-    for t in w.ctx_lens:
-        k = orc.anchor_count(t, w.ratio)
-        e += k * (k + 1) // 2
-    return e
+def run_rank_selftest(args):
+    """The multi-rank plumbing of the benchmark with a stand-in for the job: every rank joins the process group
+    (NCCL on GPUs, gloo where there is none), "runs" for 10 + 5 x rank milliseconds, and rank 0 prints the line with
+    the slowest rank's time and the whole-job value.  Exercised by the CPU tests through the same launcher
+    `--gpus N` uses."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", 0)); world = int(os.environ.get("WORLD_SIZE", 1))
+    use_cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))) if use_cuda else torch.device("cpu")
+    if use_cuda:
+        torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl" if use_cuda else "gloo")
+    ms = max_over_ranks(10.0 + 5.0 * rank, device, world)
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "ms_per_step": ms,
+                          "value": whole_job_value(2.0e12, world, ms), "backend": "nccl" if use_cuda else "gloo"}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def main():
@@ -636,28 +966,38 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="qwen14b_32k", choices=["qwen14b_32k", "llama8b_16k", "tiny", "ragged8"])
+    ap.add_argument("--workload", default="qwen14b_32k", choices=["qwen14b_32k", "llama8b_16k", "llama8b_8k", "tiny", "ragged8"])
     ap.add_argument("--variant", default="calibrated", choices=["calibrated", "literal"])
     ap.add_argument("--ratio", type=float, default=0.15)
     ap.add_argument("--layers", type=int, default=0)
     ap.add_argument("--full-prefix", action="store_true", help="Full-Prefix Control: same targets, context = every j <= p")
+    ap.add_argument("--config", default="relaxkv", choices=("relaxkv",) + LIST_CONFIGS,
+                    help="controlled configurations of the paper's appendix on the explicit-list entry points")
+    ap.add_argument("--rg", type=float, default=0.2, help="global repair target ratio of --config target_sweep")
     ap.add_argument("--dense", action="store_true",
                     help="run the whole repair loop of Algorithm 1 including the active rows' block work (projections, "
                          "rotary embedding, MLP with synthetic weights); prints its own JSON line")
     ap.add_argument("--query-attention", action="store_true",
                     help="time the user query's prefill rows and a decode step over the context cache (same kernel, context split)")
-    ap.add_argument("--attn-variant", type=int, default=0, choices=[0, 1, 2],
-                    help="attention kernel for head_dim 128: 0 two tiles per block (default), 1 SM pairs, 2 one tile with split keys")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the other benchmark configurations after the headline workload")
     ap.add_argument("--cpu-rows", type=int, default=256)
+    ap.add_argument("--selftest-ranks", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # no launcher around us: start the ranks ourselves, one process per GPU
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.selftest_ranks:
+        run_rank_selftest(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.query_attention:
         run_query_attention(args)
     elif args.dense:
         run_dense(args)
+    elif args.config != "relaxkv":
+        run_list_config(args)
     else:
         run_gpu(args)
 

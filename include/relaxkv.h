@@ -56,6 +56,15 @@ typedef enum {
 /* A CUDA stream handle (cudaStream_t) passed as an opaque pointer; NULL is the default stream. */
 typedef void* relaxkv_stream;
 
+/* Optional per-call overrides of choices the library otherwise makes from the size of the launch.  Every field:
+ * 0 = automatic.  Meant for tests and measurements; results agree within the tolerances either way. */
+typedef struct {
+  int32_t attention_ctx_splits;  /* > 0: the attention calls split every query tile's context over this many thread   */
+                                 /* blocks (up to 32, and as far as the workspace's 2048 row-splits allow) and merge   */
+                                 /* the partial results by their log-sum-exp; automatic = only when the call has too   */
+                                 /* few query tiles to fill the GPU (a query prefill, a decode step, few targets)      */
+} relaxkv_tuning;
+
 /* Shapes shared by all calls. */
 typedef struct {
   int32_t n_req;              /* 1 <= B <= 64 requests in the batch                             */
@@ -66,6 +75,7 @@ typedef struct {
   const int32_t* h_q_len;     /* host [B]: query-suffix tokens Q of each request; read by       */
                               /* relaxkv_score_select and relaxkv_workspace_bytes only          */
   float softmax_scale;        /* multiplies q.k before the softmax (usually 1/sqrt(D))          */
+  const relaxkv_tuning* h_tuning;  /* host, optional: NULL = every choice automatic             */
 } relaxkv_shape;
 
 /* One layer's KV cache.  Element (request b, token i, kv head g, dim d) of K lives at
@@ -280,6 +290,36 @@ relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers,
                                    float* mean_out, relaxkv_stream stream);
 
 /*
+ * The user query's own attention at one layer with the context scores taken from the same pass (Section 2,
+ * "running the query against the cached keys produces query-to-context attention at every layer"; Section 3.2, score
+ * equation with the row normalisers of the query's real forward pass, whose softmax also spans the query's own
+ * tokens).  For a serving caller this replaces relaxkv_score_select's scoring for the layer: the statistics pass
+ * never runs, the scores come out of the forward pass the query makes anyway.
+ *
+ * For request b the cache holds the T_c = h_ctx_len[b] context rows followed by the Q_b = h_q_len[b] rows of the
+ * query's own K/V (positions T_c .. T_c + Q_b - 1); it must hold h_req_token_offset[b] + T_c + Q_b token rows.
+ *   out[t,h,:] = causal attention of query token t (position T_c + t) over positions 0 .. T_c + t of its request
+ *   lse[h,t]   = log-normaliser of that row (context keys and the query's own keys up to t)
+ *   raw[i]     = (1/(H*Q_b)) * sum_h sum_t exp(softmax_scale * <q[t,h,:], K[i,h/G,:]> - lse[h,t])      for i < T_c
+ * q / out         device bf16 [sum_b Q_b, H, D]; lse_out device fp32 [H, sum_b Q_b] (required)
+ * raw_scores_out  device fp32 [sum_b T_c], or NULL for the attention alone.  Stack the layers' rows and feed them to
+ *                 relaxkv_select_topk for the anchors.
+ * workspace       at least relaxkv_workspace_bytes() of the same shape with h_ctx_len[b] = T_c + Q_b.
+ * Runs the cache-only attention kernel (which leaves the rows' normalisers), then the column-sum pass of the scoring
+ * kernel over the context keys with those normalisers.
+ */
+relaxkv_status relaxkv_query_prefill_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q, void* out, float* lse_out,
+    float* raw_scores_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream);
+
+/* scores[l, i] *= factor, in place, for device fp32 [n_layers, sum_b T_c] (factor > 0).  Section 3.2's score is a mean
+ * over all H query heads; when the heads are sharded over N devices of equal share, every device scores its own heads
+ * (relaxkv_score_select with anchors_out = NULL), the devices' scores are summed by one all-reduce and this call with
+ * factor = 1/N turns the sum of the shard means into the mean over all heads; relaxkv_select_topk follows. */
+relaxkv_status relaxkv_scale_scores(const relaxkv_shape* shape, int32_t n_layers, float* scores, float factor,
+                                    relaxkv_stream stream);
+
+/*
  * ---- Dense block work of the active targets (Algorithm 1, steps 14, 16 and 20; Section 3.3 for the
  * position IDs).  The method runs "the unchanged Transformer block" on the |R_l| active rows only; these
  * calls are that block for a Llama-style pre-norm decoder.  All tensors bf16, row-major, 16-byte aligned,
@@ -291,7 +331,9 @@ relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64
                                float eps, relaxkv_stream stream);
 
 /* y = x weight^T (+ residual)      x [n_rows, n_in], weight [n_out, n_in] (the [out, in] layout),
- * residual NULL or [n_rows, n_out], y [n_rows, n_out] (may alias residual).  tcgen05 GEMM. */
+ * residual NULL or [n_rows, n_out], y [n_rows, n_out] (may alias residual).  tcgen05 GEMM; calls of one to four
+ * rows (a decode token, the row that goes through the output head) stream the weights once through a plain
+ * HBM-bound kernel instead. */
 relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
                               int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream);
 
@@ -360,33 +402,6 @@ relaxkv_status relaxkv_cache_attention(
     const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q_new,
     const int32_t* tgt_pos, const int32_t* tgt_cu, int64_t n_target_rows, const int32_t* h_max_targets,
     void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream);
-
-/*
- * Test utility (the paper has no counterpart).  The attention calls split every query tile's context over
- * several thread blocks when there are too few query tiles to fill the GPU (a query prefill, a decode step, a
- * layer with few active targets) and merge the partial results by their log-sum-exp; the split count is
- * chosen from the launch size.  n_splits > 0 forces that count (up to 32, and as far as the workspace's
- * 2048 row-splits allow) for every later call of this process, 0 restores the automatic choice.
- */
-relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits);
-
-/*
- * Test utility (the paper has no counterpart).  Chooses the kernel every later attention call of this process
- * with head_dim 128 runs (head_dim 64 always runs variant 0); results agree within the attention tolerance.
- *   0  two query tiles per thread block in ping-pong (default)
- *   1  SM pairs: clusters of two blocks whose tensor cores are driven by one instruction stream, each block
- *      staging half of every K/V tile
- *   2  one query tile per block, S and P double-buffered in tensor memory, the two softmax warpgroups splitting
- *      the keys of every tile
- */
-relaxkv_status relaxkv_debug_set_attention_variant(int32_t variant);
-
-/*
- * Test utility (the paper has no counterpart).  relaxkv_linear / relaxkv_linear_swiglu run on SM pairs (clusters of
- * two thread blocks, 256 x 256 tiles, one MMA instruction stream for both tensor cores); on != 0 makes every later
- * call of this process use the single-block kernel (128 x 256 tiles), 0 restores the default.  Same results.
- */
-relaxkv_status relaxkv_debug_set_gemm_single_cta(int32_t on);
 
 /*
  * Test utility for the bounded waits (the paper has no counterpart): launches one thread that waits on

@@ -23,9 +23,9 @@ ENTRY_POINTS = (
     "relaxkv_status_string", "relaxkv_anchor_count", "relaxkv_workspace_bytes", "relaxkv_score_select",
     "relaxkv_build_active_sets", "relaxkv_sparse_ctx_attention", "relaxkv_scatter_kv", "relaxkv_gather_kv",
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
-    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout", "relaxkv_debug_set_attention_splits", "relaxkv_debug_set_attention_variant", "relaxkv_debug_set_gemm_single_cta",
+    "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
     "relaxkv_list_attention", "relaxkv_cache_attention",
-    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_swiglu", "relaxkv_rope",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_swiglu", "relaxkv_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
 
@@ -36,10 +36,15 @@ class RelaxKVError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} (status {status})")
 
 
+class _Tuning(ctypes.Structure):
+    _fields_ = [("attention_ctx_splits", ctypes.c_int32)]
+
+
 class _Shape(ctypes.Structure):
     _fields_ = [("n_req", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("h_ctx_len", ctypes.POINTER(ctypes.c_int32)),
-                ("h_q_len", ctypes.POINTER(ctypes.c_int32)), ("softmax_scale", ctypes.c_float)]
+                ("h_q_len", ctypes.POINTER(ctypes.c_int32)), ("softmax_scale", ctypes.c_float),
+                ("h_tuning", ctypes.POINTER(_Tuning))]
 
 
 class _CacheView(ctypes.Structure):
@@ -99,7 +104,8 @@ class Shape:
     """Host-side relaxkv_shape; keeps its arrays alive."""
 
     def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, ctx_lens: Sequence[int],
-                 q_lens: Optional[Sequence[int]] = None, softmax_scale: Optional[float] = None):
+                 q_lens: Optional[Sequence[int]] = None, softmax_scale: Optional[float] = None,
+                 attention_ctx_splits: int = 0):
         self.ctx_lens = [int(x) for x in ctx_lens]
         self.q_lens = None if q_lens is None else [int(x) for x in q_lens]
         self._ctx = _i32(self.ctx_lens)
@@ -110,6 +116,17 @@ class Shape:
         self.c.h_ctx_len = ctypes.cast(self._ctx, ctypes.POINTER(ctypes.c_int32))
         self.c.h_q_len = ctypes.cast(self._q, ctypes.POINTER(ctypes.c_int32)) if self._q is not None else None
         self.c.softmax_scale = float(softmax_scale if softmax_scale is not None else head_dim ** -0.5)
+        self._tuning = None
+        self.set_tuning(attention_ctx_splits)
+
+    def set_tuning(self, attention_ctx_splits: int = 0) -> None:
+        """relaxkv_tuning of the calls made with this shape (0 = the library's automatic choice)."""
+        if attention_ctx_splits:
+            self._tuning = _Tuning(int(attention_ctx_splits))
+            self.c.h_tuning = ctypes.pointer(self._tuning)
+        else:
+            self._tuning = None
+            self.c.h_tuning = None
 
     @property
     def n_req(self) -> int:
@@ -264,6 +281,16 @@ def relaxkv_cache_attention(shape: Shape, cache: CacheView, q_new: torch.Tensor,
            "relaxkv_cache_attention")
 
 
+def relaxkv_query_prefill_attention(shape: Shape, cache: CacheView, q: torch.Tensor, out: torch.Tensor, lse_out: torch.Tensor,
+                                    raw_scores_out: Optional[torch.Tensor], workspace: torch.Tensor, stream=None) -> None:
+    """shape.ctx_lens = context tokens, shape.q_lens = query tokens; the cache holds both (context rows first)."""
+    _check(lib().relaxkv_query_prefill_attention(shape.ref(), cache.ref(), _ptr(q), _ptr(out), _ptr(lse_out),
+                                                 _ptr(raw_scores_out), _ptr(workspace),
+                                                 ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                                 _stream(stream)),
+           "relaxkv_query_prefill_attention")
+
+
 def relaxkv_scatter_kv_lists(shape: Shape, cache: CacheView, k_new: torch.Tensor, v_new: torch.Tensor,
                              tgt_pos: torch.Tensor, tgt_cu: torch.Tensor, max_targets: Sequence[int], stream=None) -> None:
     _check(lib().relaxkv_scatter_kv_lists(shape.ref(), cache.ref(), _ptr(k_new), _ptr(v_new), _ptr(tgt_pos), _ptr(tgt_cu),
@@ -273,6 +300,12 @@ def relaxkv_scatter_kv_lists(shape: Shape, cache: CacheView, k_new: torch.Tensor
 def relaxkv_mean_scores(shape: Shape, n_layers: int, scores: torch.Tensor, mean_out: torch.Tensor, stream=None) -> None:
     _check(lib().relaxkv_mean_scores(shape.ref(), int(n_layers), _ptr(scores), _ptr(mean_out), _stream(stream)),
            "relaxkv_mean_scores")
+
+
+def relaxkv_scale_scores(shape: Shape, n_layers: int, scores: torch.Tensor, factor: float, stream=None) -> None:
+    """scores *= factor in place (fp32 [n_layers, sum T_c] on the device)."""
+    _check(lib().relaxkv_scale_scores(shape.ref(), int(n_layers), _ptr(scores), ctypes.c_float(factor), _stream(stream)),
+           "relaxkv_scale_scores")
 
 
 def relaxkv_rmsnorm(x: torch.Tensor, weight: torch.Tensor, y: torch.Tensor, eps: float, stream=None) -> None:
@@ -327,22 +360,6 @@ def relaxkv_carry_rows(shape: Shape, h_in: torch.Tensor, h_out: torch.Tensor, r_
     _check(lib().relaxkv_carry_rows(shape.ref(), _ptr(h_in), _ptr(h_out), int(h_in.shape[1]), _ptr(r_rank),
                                     _ptr(r_cu_layer), _ptr(r_cu_next), _i32(max_next), _stream(stream)),
            "relaxkv_carry_rows")
-
-
-def relaxkv_debug_set_attention_splits(n_splits: int) -> None:
-    """Force the attention calls' context split count (0 = chosen from the launch size).  Test hook."""
-    _check(lib().relaxkv_debug_set_attention_splits(ctypes.c_int32(int(n_splits))), "relaxkv_debug_set_attention_splits")
-
-
-def relaxkv_debug_set_attention_variant(variant: int) -> None:
-    """Kernel of head_dim-128 attention calls: 0 two tiles per block (default), 1 SM pairs, 2 one tile with split keys.
-    Test hook."""
-    _check(lib().relaxkv_debug_set_attention_variant(ctypes.c_int32(int(variant))), "relaxkv_debug_set_attention_variant")
-
-
-def relaxkv_debug_set_gemm_single_cta(on: bool) -> None:
-    """Run the GEMM calls on the single-block kernel instead of SM pairs (the default).  Test hook."""
-    _check(lib().relaxkv_debug_set_gemm_single_cta(ctypes.c_int32(1 if on else 0)), "relaxkv_debug_set_gemm_single_cta")
 
 
 def relaxkv_debug_wait_timeout(stream=None) -> None:

@@ -10,15 +10,29 @@ __device__ DeviceStatus g_status_word;
 
 DeviceStatus* status_word() {
   // One lookup per device; the address of a __device__ variable differs between devices.
-  static DeviceStatus* cached[64] = {nullptr};
+  static std::atomic<DeviceStatus*> cached[kMaxDevices];
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!cached[dev]) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-    cached[dev] = static_cast<DeviceStatus*>(p);
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceStatus* p = cached[dev].load(std::memory_order_acquire);
+  if (!p) {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_status_word) != cudaSuccess) return nullptr;
+    p = static_cast<DeviceStatus*>(q);
+    cached[dev].store(p, std::memory_order_release);
   }
-  return cached[dev];
+  return p;
+}
+
+int sm_count_of_current_device() {
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  int n = cached[dev].load(std::memory_order_acquire);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 0;
+    cached[dev].store(n, std::memory_order_release);
+  }
+  return n;
 }
 
 }  // namespace relaxkv

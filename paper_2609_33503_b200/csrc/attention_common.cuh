@@ -67,7 +67,7 @@ inline relaxkv_status prepare_attention(
   plan.kv_token_stride_bytes = (unsigned long long)shape->n_kv_heads * shape->head_dim * 2;
   plan.dense_ctx = 0;
   return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, fresh_row,
-                       need_ctx + kCtxPadRows, plan.kctx, plan.vctx, plan.ctx_rows, stream);
+                       fresh_row ? need_ctx : 0, n_target_rows, need_ctx + kCtxPadRows, plan.kctx, plan.vctx, plan.ctx_rows, stream);
 }
 
 }  // namespace relaxkv

@@ -10,8 +10,9 @@
 // A CTA runs TWO such query tiles (A, B) in ping-pong: while the softmax warps of one tile work, the
 // tensor pipe runs the other tile's MMAs; both tiles share every K/V tile staged in shared memory.
 // Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = query row = TMEM
-// lane), warp 8 TMA producer, warp 9 MMA issuer and TMEM owner.  K/V tiles move through a 5-slot ring in the
-// order K_0 V_0 K_1 V_1 ... and are signalled in pairs (V_j, K_{j+1}) - what step j of the MMA warp consumes.
+// lane), warp 8 TMA producer, warp 9 MMA issuer and TMEM owner, warp 10 a helper for cache-only calls.  K/V tiles
+// move through a 5-slot ring in the order K_0 V_0 K_1 V_1 ... and are signalled in pairs (V_j, K_{j+1}) - what
+// step j of the MMA warp consumes.
 // When a call has too few query tiles to fill the GPU, grid.y splits every pair's context; the blocks leave
 // normalised partial results that combine_splits_kernel merges by their log-sum-exp.  The K/V tensor maps
 // cover either the materialised mixed context (the repair calls) or the cache itself (relaxkv_cache_attention).
@@ -20,6 +21,7 @@
 #include "attention_common.cuh"
 #include "sm100_ptx.cuh"
 #include <algorithm>
+#include <atomic>
 
 namespace relaxkv {
 
@@ -43,7 +45,7 @@ struct AttnSmem {
   static constexpr int kKV = kQ + 2 * kTileBytes;               // ring of kRing K/V tiles
   static constexpr int kBar = kKV + kRing * kTileBytes;         // mbarriers (8 B each)
   static constexpr int kPairBars = 3;                           // (V_j, K_{j+1}) pairs in flight: full and empty barriers
-  static constexpr int kNumBars = 1 + 8 + 2 * kPairBars;
+  static constexpr int kNumBars = 1 + 8 + 2 * kPairBars + 2;
   static constexpr int kMisc = kBar + 8 * kNumBars;             // tmem address, abort flag
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                // slack to align the base to 1024 B
@@ -80,7 +82,9 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int pair_targets = 2 * tile_targets;
   const int n_pairs_true = (nr + pair_targets - 1) / pair_targets;
   if (p_rev >= n_pairs_true) return;
-  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b])) {
+  // a true count above its host bound, or more target rows than q_new / out hold: report, touch nothing
+  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b]) ||
+      (long long)(r_cu[b + 1] - r_cu[0]) > n_target_rows) {
     if (threadIdx.x == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
     return;
   }
@@ -125,6 +129,12 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     return;
   }
 
+  // Cache-only calls read K/V tiles straight from the cache: the last tile of a request may reach past the request's
+  // final token into rows that belong to nobody.  Their keys are masked, but their V rows would still meet a zero
+  // probability on the tensor core (0 x NaN = NaN), so a helper warp zeroes those V rows once the tile has landed.
+  const int v_fix_tile = (dense_ctx && (ctx_len_b % kBN) != 0) ? (ctx_len_b / kBN - j0) : -1;
+  const bool need_v_fix = v_fix_tile >= 0 && v_fix_tile < n_my_max;
+
   // ---- shared memory -----------------------------------------------------------------------------
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -138,6 +148,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_ofinal = bar0 + 56;        // [2]
   const uint32_t bar_full = bar0 + 72;          // [kPairBars] pair p = (V_{p-1}, K_p) has landed
   const uint32_t bar_empty = bar_full + 8 * L::kPairBars;   // [kPairBars] pair p has been consumed by both tiles
+  const uint32_t bar_vreq = bar_empty + 8 * L::kPairBars;   // the request's last V tile has landed (MMA warp -> helper warp)
+  const uint32_t bar_vfix = bar_vreq + 8;                   // its rows past the request's end are zeroed (helper -> MMA warp)
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
 
@@ -147,6 +159,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     mbar_init(bar_q, 1);
     for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_pfull_hi + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
     for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_vreq, 1);
+    mbar_init(bar_vfix, 32);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -244,6 +258,10 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0; this step consumes pair j + 1
         const int pr = j + 1;
         if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
+        if (need_v_fix && j == v_fix_tile) {                    // V_j reaches past the request's end: have those rows zeroed
+          mbar_arrive(bar_vreq);
+          if (!(ok = mbar_wait(bar_vfix, 0, abort_flag))) break;
+        }
         tc_fence_after();
         if (j < n_my[0]) {
           if (!(ok = issue_pv(0, j))) break;
@@ -256,6 +274,18 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         mma_commit(bar_empty + 8 * (pr % L::kPairBars));        // V_j and K_{j+1}: free once both tiles are through
       }
     }
+  } else if (warp == 10 && need_v_fix) {
+    // ================= helper: zero the V rows past the request's last token (cache-only calls) =================
+    if (mbar_wait(bar_vreq, 0, abort_flag)) {                   // raised by the MMA warp once that tile has landed
+      const int first = ctx_len_b % kBN;                        // first foreign row of the tile
+      uint8_t* vt = base_ptr + L::kKV + ((2 * v_fix_tile + 1) % kRing) * L::kTileBytes;
+      for (int i = lane; i < (kBN - first) * 8 * kHalves; i += 32) {
+        const int piece = i & 7, r = first + ((i >> 3) % (kBN - first)), hf = (i >> 3) / (kBN - first);
+        *reinterpret_cast<uint4*>(vt + hf * kHalfBytes + r * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
+      }
+      fence_proxy_async_smem();
+    }
+    mbar_arrive(bar_vfix);
   }
   } else {
     reg_alloc<224>();
@@ -442,834 +472,6 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   }
 }
 
-// ---- the same kernel for a PAIR of SMs (cta_group::2, head_dim 128) ----------------------------------------------------
-// A cluster of two CTAs walks one context for four query tiles.  One thread of the leader CTA issues every MMA with
-// M = 256 (tile x of both CTAs at once), so the per-SM cost of issuing halves, and each CTA stages only half of every
-// K/V tile (the B operand is split over the pair along N), which halves the L2 -> shared-memory traffic.  Softmax,
-// masking, the P hand-over and the epilogue are those of the single-CTA kernel; hand-overs that cross the CTA
-// boundary use cluster-scope mbarrier arrivals (peer -> leader) and multicast commits (leader -> both).
-struct PairSmem {
-  static constexpr int kQTileBytes = 2 * kHalfBytes;              // a 128 x 128 query tile
-  static constexpr int kKvTileBytes = kHalfBytes;                 // this CTA's half of a K or V tile
-  static constexpr int kPairBars = 4;                             // (V_j, K_{j+1}) pairs in flight
-  static constexpr int kRing = 2 * kPairBars;                     // ring slots
-  static constexpr int kQ = 0;
-  static constexpr int kKV = kQ + 2 * kQTileBytes;
-  static constexpr int kBar = kKV + kRing * kKvTileBytes;
-  static constexpr int kNumBars = 1 + 8 + 2 * kPairBars;
-  static constexpr int kMisc = kBar + 8 * kNumBars;
-  static constexpr int kTotal = kMisc + 16;
-  static constexpr int kDynamic = kTotal + 1024;
-};
-
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
-attention_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
-                       int mode, int allow_empty, int head_inner, int dense_ctx, int H, int Hkv, int tile_targets, float scale_log2,
-                       const int* __restrict__ u_pos, const int* __restrict__ u_cu,
-                       const int* __restrict__ r_rank, const int* __restrict__ r_cu,
-                       long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
-                       float* __restrict__ part_o, float* __restrict__ part_lse, DeviceStatus* st) {
-  using L = PairSmem;
-  constexpr int D = 128;
-  constexpr int kHalves = 2;
-  constexpr uint32_t kTmemCols = 512;          // S_A | S_B | O_A | O_B, 128 columns each (O uses D of them)
-
-  // ---- which tile pairs -------------------------------------------------------------------------------
-  // A cluster of two CTAs (an SM pair) walks the same context for FOUR query tiles: CTA rank 0 (the leader, which
-  // issues every MMA for both SMs) owns the pair with the longer context, rank 1 the next one.  rt.tile_cu counts
-  // CLUSTERS per request (from the host bounds); they are walked from the end of the target list.
-  const uint32_t cr = cluster_ctarank();
-  const int B = rt.n_req;
-  const int G = H / Hkv;
-  const int n_cl_total = rt.tile_cu[B];
-  const int cidx = (int)(blockIdx.x >> 1);
-  const int hd = head_inner ? (cidx % Hkv) : (cidx / n_cl_total);
-  const int tt = head_inner ? (cidx / Hkv) : (cidx - hd * n_cl_total);
-  const int b = find_segment(rt.tile_cu, B, tt);
-  const int c_rev = tt - rt.tile_cu[b];
-  const int nr = r_cu[b + 1] - r_cu[b];
-  // dense_ctx: the context is the cache itself (every position of the request), a target's limit is its position
-  const int nu = dense_ctx ? rt.ctx_len[b] : (u_cu[b + 1] - u_cu[b]);
-  const int pair_targets = 2 * tile_targets;
-  const int n_pairs_true = (nr + pair_targets - 1) / pair_targets;
-  if (2 * c_rev >= n_pairs_true) return;                       // the same for both CTAs of the cluster
-  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b])) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
-    return;
-  }
-  // (no early drain after a timeout here: the two CTAs of a cluster must take every exit together)
-  const int ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
-  const long long ctx_base = dense_ctx ? rt.tok_off[b] : ((mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b]);
-  // valid targets and context tiles of the four query tiles (both CTAs compute all of them: the step counts of
-  // the cluster are the maxima over its two CTAs, because one MMA instruction serves tile x of both)
-  int n_valid[2] = {0, 0}, n_step[2] = {0, 0};
-  int rho0 = 0;
-#pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
-    const int pr_ = n_pairs_true - 1 - (2 * c_rev + rr);       // -1: the peer of the last cluster has no targets
-    const int rho_r = max(pr_, 0) * pair_targets;
-    if (rr == (int)cr) rho0 = rho_r;
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-      const int nv = (pr_ < 0) ? 0 : max(0, min(tile_targets, nr - rho_r - x * tile_targets));
-      int nk = 0;
-      if (nv > 0) {
-        const int c = r_rank[r_cu[b] + rho_r + x * tile_targets + nv - 1];
-        const int cc = min(max(c, 0), max(nu - 1, 0));
-        int lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[u_cu[b] + cc];
-        lim_last = min(max(lim_last, 0), ctx_len_b - 1);
-        nk = lim_last / kBN + 1;
-      }
-      if (rr == (int)cr) n_valid[x] = nv;
-      n_step[x] = max(n_step[x], nk);
-    }
-  }
-  const long long q_row_base = (long long)(r_cu[b] - r_cu[0]) + rho0;
-  const int n_kv_max = max(n_step[0], n_step[1]);
-  // Context split (gridDim.y > 1): this cluster walks the context tiles [j0, j0 + chunk) of its tiles.
-  const int n_splits = (int)gridDim.y, split = (int)blockIdx.y;
-  const int chunk = (n_kv_max + n_splits - 1) / n_splits;
-  const int j0 = split * chunk;
-  int n_my[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) n_my[x] = max(0, min(n_step[x], j0 + chunk) - j0);
-  const int n_my_max = max(n_my[0], n_my[1]);
-  if (n_my_max == 0) {                        // nothing of this cluster's context falls into this split (both CTAs)
-    if (n_splits > 1 && threadIdx.x < 2 * kBM) {
-      const int x = threadIdx.x >> 7, row = threadIdx.x & 127, t_local = row / G;
-      if (row < tile_targets * G && t_local < n_valid[x]) {
-        const long long orow = q_row_base + x * tile_targets + t_local;
-        part_lse[((long long)split * n_target_rows + orow) * H + hd * G + (row - t_local * G)] = -INFINITY;
-      }
-    }
-    return;
-  }
-
-  // ---- shared memory -----------------------------------------------------------------------------
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base + L::kQ, kv_smem = base + L::kKV;
-  const uint32_t bar0 = base + L::kBar;
-  const uint32_t bar_q = bar0;
-  const uint32_t bar_sfull = bar0 + 8;          // [2]
-  const uint32_t bar_pfull = bar0 + 24;         // [2] first 64 keys of P ready
-  const uint32_t bar_pfull_hi = bar0 + 40;      // [2] last 64 keys of P ready
-  const uint32_t bar_ofinal = bar0 + 56;        // [2]
-  const uint32_t bar_full = bar0 + 72;          // [kPairBars] pair p = (V_{p-1}, K_p) has landed (leader: in both CTAs)
-  const uint32_t bar_empty = bar_full + 8 * L::kPairBars;   // [kPairBars] pair p has been consumed by both tiles
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    // The leader's "data has landed" barriers also count one arrival relayed from the peer CTA, and its P barriers
-    // the 128 softmax threads of each CTA; the peer's copies of the P barriers are not used.
-    const uint32_t n_cta = (cr == 0) ? 2u : 1u;
-    mbar_init(bar_q, n_cta);
-    for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 256); mbar_init(bar_pfull_hi + 8 * x, 256); mbar_init(bar_ofinal + 8 * x, 1); }
-    for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, n_cta); mbar_init(bar_empty + 8 * s, 1); }
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async_smem();
-  }
-  if (warp == 9) {
-    tmem_alloc2(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);      // one warp of EACH CTA of the pair
-    tmem_relinquish2();
-  }
-  // rows of the Q tiles that no (target, head) pair fills: zero them (they feed unused MMA rows)
-  {
-    const int used = tile_targets * G;
-    const int n_pad = kBM - used;
-    for (int i = threadIdx.x; i < n_pad * 8 * kHalves * 2; i += kAttnThreads) {
-      const int piece = i & 7, r = (i >> 3) % n_pad, blk = (i >> 3) / n_pad;    // blk = tile * kHalves + half
-      *reinterpret_cast<uint4*>(base_ptr + L::kQ + blk * kHalfBytes + (used + r) * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
-    }
-    fence_proxy_async_smem();
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync();                             // both CTAs: barriers initialised, TMEM allocated, padding rows written
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  // Register budget: the control warpgroup gives registers to the two softmax warpgroups
-  // (12 warps x 168 at launch = 8 x 224 + 4 x 56).
-  if (warp >= 8) {
-  reg_dealloc<56>();
-  if (warp == 8) {
-    // ================= TMA producer =================
-    if (lane == 0) {
-      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      mbar_expect_tx(bar_q, (uint32_t)(2 * kHalves * tile_targets * G * 128));
-      for (int x = 0; x < 2; ++x)
-        for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_3d(q_smem + (x * kHalves + hf) * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G,
-                      (int)(q_row_base + x * tile_targets));
-      // The tiles travel in the order K_0 V_0 K_1 V_1 ... through the ring slots u % L::kRing (u = 2j for K_j, 2j + 1
-      // for V_j; j counted from j0) and are signalled in PAIRS p = (V_{p-1}, K_p), what step p - 1 of the MMA warp
-      // consumes.  This CTA stages only ITS HALF of every tile: the B operand of a cta_group::2 MMA is split over
-      // the two CTAs along N - keys [64 cr, 64 cr + 64) of a K tile, head-dim columns [64 cr, 64 cr + 64) of a V tile.
-      auto load_tile = [&](int u, uint32_t bar) {
-        const int s = u % L::kRing;
-        const int row = (int)(ctx_base + (long long)(j0 + (u >> 1)) * kBN);
-        const uint32_t dst = kv_smem + s * L::kKvTileBytes;
-        if (u & 1) {
-          tma_load_3d(dst, &tm_v, bar, 64 * (int)cr, hd, row);                       // 128 keys x 64 columns
-        } else {
-          for (int hf = 0; hf < kHalves; ++hf)                                         // 64 keys x (64 + 64) columns
-            tma_load_3d(dst + hf * (L::kKvTileBytes / 2), &tm_k, bar, hf * 64, hd, row + 64 * (int)cr);
-        }
-      };
-      for (int pr = 0; pr <= n_my_max; ++pr) {                  // pair pr: V_{pr-1} (if pr > 0) and K_pr (if pr < n)
-        const uint32_t bar = bar_full + 8 * (pr % L::kPairBars);
-        const bool has_v = pr > 0, has_k = pr < n_my_max;
-        // both slots were last used by pair pr - kPairBars (ring of 2 * kPairBars slots)
-        if (pr >= L::kPairBars &&
-            !mbar_wait(bar_empty + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(bar, (uint32_t)((has_v ? L::kKvTileBytes : 0) + (has_k ? L::kKvTileBytes : 0)));
-        if (has_v) load_tile(2 * pr - 1, bar);
-        if (has_k) load_tile(2 * pr, bar);
-      }
-    }
-  } else if (warp == 9) {
-    // ================= leader CTA: MMA issuer for both SMs; peer CTA: relays "my half has landed" =================
-    if (lane == 0 && cr != 0) {
-      // the leader's "landed" barriers wait for this CTA's copies too: forward each completion with one remote arrival
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
-      if (ok) mbar_arrive_remote(mapa_shared(bar_q, 0));
-      for (int pr = 0; ok && pr <= n_my_max; ++pr) {
-        if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
-        mbar_arrive_remote(mapa_shared(bar_full + 8 * (pr % L::kPairBars), 0));
-      }
-    }
-    if (lane == 0 && cr == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(2 * kBM, kBN, 0);       // M = 256: tile x of both CTAs
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(2 * kBM, D, 1);
-      bool ok = mbar_wait_cluster(bar_q, 0, abort_flag);
-      // S_x = Q_x K_j^T  -> bar_sfull[x] of both CTAs
-      auto issue_qk = [&](int x, int j) {
-        const int s = (2 * j) % L::kRing;
-        mma2_ss_kloop(tmem_base + x * 128, desc_lo(q_smem + x * L::kQTileBytes, 16),
-                      desc_lo(kv_smem + s * L::kKvTileBytes, 16), desc_hi_sw128(1024), idesc_qk);
-        mma_commit2_mc(bar_sfull + 8 * x, 3);
-      };
-      // O_x += P_x V_j   (P_x read from each CTA's TMEM where its softmax warps left it, over S_x)
-      auto issue_pv = [&](int x, int j) -> bool {
-        const int s = (2 * j + 1) % L::kRing;
-        if (!mbar_wait_cluster(bar_pfull + 8 * x, j & 1, abort_flag)) return false;
-        tc_fence_after();
-        const uint32_t v_lo = desc_lo(kv_smem + s * L::kKvTileBytes, L::kKvTileBytes);
-        mma2_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128, v_lo, desc_hi_sw128(1024), idesc_pv, j > 0 ? 1u : 0u);
-        // the second half of P arrives while the first half is being multiplied
-        if (!mbar_wait_cluster(bar_pfull_hi + 8 * x, j & 1, abort_flag)) return false;
-        tc_fence_after();
-        mma2_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128 + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
-        if (j == n_my[x] - 1) mma_commit2_mc(bar_ofinal + 8 * x, 3);
-        return true;
-      };
-      // pair 0 = K_0 alone
-      if (ok) ok = mbar_wait_cluster(bar_full, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        if (n_my[0] > 0) issue_qk(0, 0);
-        if (n_my[1] > 0) issue_qk(1, 0);
-        mma_commit2_mc(bar_empty, 3);
-      }
-      for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0; this step consumes pair j + 1
-        const int pr = j + 1;
-        if (!(ok = mbar_wait_cluster(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
-        tc_fence_after();
-        if (j < n_my[0]) {
-          if (!(ok = issue_pv(0, j))) break;
-          if (j + 1 < n_my[0]) issue_qk(0, j + 1);
-        }
-        if (j < n_my[1]) {
-          if (!(ok = issue_pv(1, j))) break;
-          if (j + 1 < n_my[1]) issue_qk(1, j + 1);
-        }
-        mma_commit2_mc(bar_empty + 8 * (pr % L::kPairBars), 3);   // V_j and K_{j+1}: free in both CTAs
-      }
-    }
-  }
-  } else {
-    reg_alloc<224>();
-    // ================= softmax + epilogue: thread = query row = TMEM lane =================
-    const int x = warp >> 2;                                    // 0: tile A, 1: tile B
-    const int row = threadIdx.x & 127;
-    const int t_local = row / G, j_head = row - t_local * G;
-    const bool row_valid = (row < tile_targets * G) && (t_local < n_valid[x]);
-    const int rho_t = rho0 + x * tile_targets + t_local;
-    int limit = 0;
-    bool row_empty = false;                                     // explicit lists: a target that sees no context entry
-    if (row_valid) {
-      const int c = r_rank[r_cu[b] + rho_t];
-      if (c == -1 && allow_empty) {
-        row_empty = true;
-      } else if (c < 0 || c >= nu) {
-        report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
-      } else {
-        limit = (mode == RELAXKV_CTX_UNION) ? c : u_pos[u_cu[b] + c];
-        if (limit < 0 || limit >= ctx_len_b) { report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, limit, ctx_len_b); limit = 0; }
-      }
-    }
-    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t t_s = lane_base + x * 128, t_o = lane_base + 256 + x * 128;
-    const uint32_t my_sfull = bar_sfull + 8 * x;
-    const uint32_t ld_pfull = mapa_shared(bar_pfull + 8 * x, 0), ld_pfull_hi = mapa_shared(bar_pfull_hi + 8 * x, 0);   // in the leader CTA
-    const int my_n = n_my[x];
-    float m = -INFINITY, z = 0.f;
-    bool ok = true;
-    for (int j = 0; j < my_n; ++j) {
-      ok = mbar_wait(my_sfull, j & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t s[kBN];
-#pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) tmem_ld32(t_s + c * 32, &s[c * 32]);
-      tmem_wait_ld();
-      const int col0 = (j0 + j) * kBN;
-      if (col0 + kBN - 1 > limit) {
-#pragma unroll
-        for (int i = 0; i < kBN; ++i)
-          if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
-      }
-      // row maximum: eight independent chains instead of one 128-deep dependency chain
-      float mx8[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
-#pragma unroll
-      for (int i = 8; i + 16 <= kBN; i += 16) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) mx8[e] = fmax3(mx8[e], __uint_as_float(s[i + e]), __uint_as_float(s[i + 8 + e]));
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[kBN - 8 + e]));
-      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-      const float m_new = mx * scale_log2;
-      if (j == 0) {
-        m = fmaxf(m_new, -1.0e30f);           // a row whose first tile of this split is fully masked keeps a finite reference
-      } else {
-        // S_x(j) is complete, hence so is O_x += P_x V_{j-1}: O_x may be rescaled here
-        const bool need = m_new > m + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          float alpha = 1.f;
-          if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(t_o + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st32(t_o + c * 32, o);
-          }
-          tmem_wait_st();
-        }
-      }
-      float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
-      const float neg_m = -m;
-#pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          // p = 2^(s * scale - m) for eight keys; the scaling and the row sums use packed fp32 pairs
-          float x[8], p[8];
-#pragma unroll
-          for (int e = 0; e < 8; e += 2)
-            fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
-                 scale_log2, neg_m, neg_m);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
-          add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
-          add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
-#pragma unroll
-          for (int e = 0; e < 8; e += 2) {
-            __nv_bfloat162 h = __floats2bfloat162_rn(p[e], p[e + 1]);
-            pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h);
-          }
-        }
-        tmem_st16(t_s + c * 16, pk);
-        if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
-          tmem_wait_st();
-          tc_fence_before();
-          if (cr == 0) mbar_arrive(bar_pfull + 8 * x); else mbar_arrive_remote(ld_pfull);
-        }
-      }
-      z += (zs0 + zs1) + (zs2 + zs3);
-      tmem_wait_st();
-      tc_fence_before();
-      if (cr == 0) mbar_arrive(bar_pfull_hi + 8 * x); else mbar_arrive_remote(ld_pfull_hi);
-    }
-    if (ok && my_n > 0) {
-      ok = mbar_wait(bar_ofinal + 8 * x, 0, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok && my_n > 0) {
-      tc_fence_after();
-      const bool none = row_empty || !(z > 0.f);                // an empty context is defined as a zero output row
-      const float inv = none ? 0.f : 1.f / z;
-      const float lse = none ? -INFINITY : (m + log2f(z)) * kLn2A;
-      const long long orow = q_row_base + x * tile_targets + t_local;
-      if (n_splits == 1) {
-        uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(t_o + c * 32, o);
-          tmem_wait_ld();
-          if (row_valid) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv,
-                                                          __uint_as_float(o[i + 2 * e + 1]) * inv);
-                w[e] = *reinterpret_cast<uint32_t*>(&h2);
-              }
-              *reinterpret_cast<uint4*>(optr + c * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-        if (row_valid && lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = lse;
-      } else {
-        // partial result of this split: fp32, normalised by this split's own sum
-        const long long slot = ((long long)split * n_target_rows + orow) * H + hd * G + j_head;
-        float* optr = part_o + slot * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(t_o + c * 32, o);
-          tmem_wait_ld();
-          if (row_valid) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              *reinterpret_cast<float4*>(optr + c * 32 + i) =
-                  make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv, __uint_as_float(o[i + 2]) * inv,
-                              __uint_as_float(o[i + 3]) * inv);
-          }
-        }
-        if (row_valid) part_lse[slot] = lse;
-      }
-    } else if (ok && my_n == 0 && n_splits > 1 && row_valid) {
-      // this tile's context ends before the split begins (the pair's other tile still has work here)
-      const long long orow = q_row_base + x * tile_targets + t_local;
-      part_lse[((long long)split * n_target_rows + orow) * H + hd * G + j_head] = -INFINITY;
-    }
-  }
-
-  // ---- teardown ------------------------------------------------------------------------------------
-  tc_fence_before();
-  __syncthreads();
-  if (*abort_flag) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, cidx, hd);
-    // give copies and MMAs still in flight time to land before shared memory and TMEM are released
-    const uint64_t t0 = global_timer_ns();
-    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
-    __syncthreads();
-  }
-  cluster_sync();                             // the peer's shared memory and TMEM are operands of the leader's MMAs
-  if (warp == 9) {
-    tc_fence_after();
-    tmem_dealloc2(tmem_base, kTmemCols);
-  }
-}
-
-// ---- one query tile per CTA, S and P double-buffered, the two softmax warpgroups split the KEYS of every tile ---------
-// TMEM: S0 | S1 (2 x 128 columns), O (128), P0 | P1 (2 x 64): with P out of S's columns and a second S buffer the MMA
-// warp issues Q K^T of step j + 1 before P V of step j, so a tile's softmax never waits for its own MMAs (in the
-// two-tile kernel above S and P share columns and every step is a dependency chain).  Thread = (query row, key half):
-// warpgroup h handles keys [64 h, 64 h + 64) of every tile; the two halves of a row agree on the reference exponent
-// through shared memory (one named barrier per step), keep partial row sums, and each rescales half of O's columns.
-struct SplitSmem {
-  static constexpr int kQTileBytes = 2 * kHalfBytes;
-  static constexpr int kTileBytes = 2 * kHalfBytes;               // a whole K or V tile
-  static constexpr int kPairBars = 3;
-  static constexpr int kRing = 2 * kPairBars;
-  static constexpr int kQ = 0;
-  static constexpr int kKV = kQ + kQTileBytes;
-  static constexpr int kXch = kKV + kRing * kTileBytes;           // float [2][128]: row maxima / row sums of the halves
-  static constexpr int kBar = kXch + 2 * 128 * 4;
-  static constexpr int kNumBars = 1 + 2 + 2 + 2 + 2 + 1 + 2 * kPairBars;   // q, sfull, sfree, pfull, pvdone, ofinal, full, empty
-  static constexpr int kMisc = kBar + 8 * kNumBars;
-  static constexpr int kTotal = kMisc + 16;
-  static constexpr int kDynamic = kTotal + 1024;
-};
-
-__device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
-}
-
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attention_split_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
-                             int mode, int allow_empty, int head_inner, int dense_ctx, int H, int Hkv, int tile_targets, float scale_log2,
-                             const int* __restrict__ u_pos, const int* __restrict__ u_cu,
-                             const int* __restrict__ r_rank, const int* __restrict__ r_cu,
-                             long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
-                             float* __restrict__ part_o, float* __restrict__ part_lse, DeviceStatus* st) {
-  using L = SplitSmem;
-  constexpr int D = 128;
-  constexpr int kHalves = 2;
-  constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
-
-  // ---- which query tile: rt.tile_cu counts TILES per request (host bounds), walked from the end of the target list ----
-  const int B = rt.n_req;
-  const int G = H / Hkv;
-  const int n_tiles_total = rt.tile_cu[B];
-  const int hd = head_inner ? (int)(blockIdx.x % Hkv) : (int)(blockIdx.x / n_tiles_total);
-  const int tt = head_inner ? (int)(blockIdx.x / Hkv) : (int)(blockIdx.x - hd * n_tiles_total);
-  const int b = find_segment(rt.tile_cu, B, tt);
-  const int t_rev = tt - rt.tile_cu[b];
-  const int nr = r_cu[b + 1] - r_cu[b];
-  const int nu = dense_ctx ? rt.ctx_len[b] : (u_cu[b + 1] - u_cu[b]);
-  const int n_tiles_true = (nr + tile_targets - 1) / tile_targets;
-  if (t_rev >= n_tiles_true) return;
-  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b])) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
-    return;
-  }
-  if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;   // drain after a timeout
-  const int tile = n_tiles_true - 1 - t_rev;
-  const int rho0 = tile * tile_targets;
-  const int ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
-  const long long ctx_base = dense_ctx ? rt.tok_off[b] : ((mode == RELAXKV_CTX_UNION) ? (long long)u_cu[b] : rt.ctx_cu[b]);
-  const long long q_row_base = (long long)(r_cu[b] - r_cu[0]) + rho0;
-  const int n_valid = max(0, min(tile_targets, nr - rho0));
-  int n_kv = 0;
-  {
-    const int c = r_rank[r_cu[b] + rho0 + n_valid - 1];
-    const int cc = min(max(c, 0), max(nu - 1, 0));
-    int lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[u_cu[b] + cc];
-    lim_last = min(max(lim_last, 0), ctx_len_b - 1);
-    n_kv = lim_last / kBN + 1;
-  }
-  const int n_splits = (int)gridDim.y, split = (int)blockIdx.y;
-  const int chunk = (n_kv + n_splits - 1) / n_splits;
-  const int j0 = split * chunk;
-  const int n_my = max(0, min(n_kv, j0 + chunk) - j0);
-  if (n_my == 0) {                            // nothing of this tile's context falls into this split
-    if (n_splits > 1 && threadIdx.x < kBM) {
-      const int row = threadIdx.x, t_local = row / G;
-      if (row < tile_targets * G && t_local < n_valid)
-        part_lse[((long long)split * n_target_rows + q_row_base + t_local) * H + hd * G + (row - t_local * G)] = -INFINITY;
-    }
-    return;
-  }
-
-  // ---- shared memory ----
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base + L::kQ, kv_smem = base + L::kKV;
-  float* xch = reinterpret_cast<float*>(base_ptr + L::kXch);
-  const uint32_t bar0 = base + L::kBar;
-  const uint32_t bar_q = bar0;
-  const uint32_t bar_sfull = bar0 + 8;          // [2] S buffer written
-  const uint32_t bar_sfree = bar0 + 24;         // [2] S buffer read into registers by all 256 softmax threads
-  const uint32_t bar_pfull = bar0 + 40;         // [2] P buffer written
-  const uint32_t bar_pvdone = bar0 + 56;        // [2] P V of the step that used this P buffer has completed
-  const uint32_t bar_ofinal = bar0 + 72;
-  const uint32_t bar_full = bar0 + 80;          // [kPairBars] pair p = (V_{p-1}, K_p) has landed
-  const uint32_t bar_empty = bar_full + 8 * L::kPairBars;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    mbar_init(bar_q, 1);
-    for (int x = 0; x < 2; ++x) {
-      mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_sfree + 8 * x, 256); mbar_init(bar_pfull + 8 * x, 256); mbar_init(bar_pvdone + 8 * x, 1);
-    }
-    mbar_init(bar_ofinal, 1);
-    for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async_smem();
-  }
-  if (warp == 9) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols); tmem_relinquish(); }
-  {
-    const int used = tile_targets * G, n_pad = kBM - used;      // rows no (target, head) pair fills: zero them
-    for (int i = threadIdx.x; i < n_pad * 8 * kHalves; i += kAttnThreads) {
-      const int piece = i & 7, r = (i >> 3) % n_pad, hf = (i >> 3) / n_pad;
-      *reinterpret_cast<uint4*>(base_ptr + L::kQ + hf * kHalfBytes + (used + r) * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
-    }
-    fence_proxy_async_smem();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp >= 8) {
-  reg_dealloc<56>();
-  if (warp == 8) {
-    // ================= TMA producer =================
-    if (lane == 0) {
-      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      mbar_expect_tx(bar_q, (uint32_t)(kHalves * tile_targets * G * 128));
-      for (int hf = 0; hf < kHalves; ++hf)
-        tma_load_3d(q_smem + hf * kHalfBytes, &tm_q, bar_q, hf * 64, hd * G, (int)q_row_base);
-      // tiles in the order K_0 V_0 K_1 V_1 ... through ring slots u % kRing, signalled in pairs p = (V_{p-1}, K_p)
-      auto load_tile = [&](int u, uint32_t bar) {
-        const int s = u % L::kRing;
-        const int row = (int)(ctx_base + (long long)(j0 + (u >> 1)) * kBN);
-        const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
-        for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar, hf * 64, hd, row);
-      };
-      for (int pr = 0; pr <= n_my; ++pr) {
-        const uint32_t bar = bar_full + 8 * (pr % L::kPairBars);
-        const bool has_v = pr > 0, has_k = pr < n_my;
-        if (pr >= L::kPairBars &&
-            !mbar_wait(bar_empty + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(bar, (uint32_t)((has_v ? L::kTileBytes : 0) + (has_k ? L::kTileBytes : 0)));
-        if (has_v) load_tile(2 * pr - 1, bar);
-        if (has_k) load_tile(2 * pr, bar);
-      }
-    }
-  } else if (warp == 9) {
-    // ================= MMA issuer =================
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(kBM, kBN, 0);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
-      auto issue_qk = [&](int j) {                              // S_{j & 1} = Q K_j^T
-        const int s = (2 * j) % L::kRing;
-        mma_ss_kloop<kHalves>(tmem_base + kColS + (j & 1) * 128, desc_lo(q_smem, 16), desc_lo(kv_smem + s * L::kTileBytes, 16),
-                              desc_hi_sw128(1024), idesc_qk);
-        mma_commit(bar_sfull + 8 * (j & 1));
-      };
-      if (ok) ok = mbar_wait(bar_full, 0, abort_flag);          // pair 0 = K_0 alone
-      if (ok) {
-        tc_fence_after();
-        issue_qk(0);
-        mma_commit(bar_empty);
-      }
-      for (int j = 0; ok && j < n_my; ++j) {                    // this step consumes pair j + 1 = (V_j, K_{j+1})
-        const int pr = j + 1;
-        if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
-        if (j + 1 < n_my) {
-          // S buffer (j + 1) & 1 was last read by the softmax of step j - 1
-          if (j >= 1 && !(ok = mbar_wait(bar_sfree + 8 * ((j + 1) & 1), (uint32_t)((j - 1) >> 1) & 1, abort_flag))) break;
-          tc_fence_after();
-          issue_qk(j + 1);
-        }
-        // O += P_j V_j   (P buffer j & 1)
-        if (!(ok = mbar_wait(bar_pfull + 8 * (j & 1), (uint32_t)(j >> 1) & 1, abort_flag))) break;
-        tc_fence_after();
-        const uint32_t v_lo = desc_lo(kv_smem + ((2 * j + 1) % L::kRing) * L::kTileBytes, kHalfBytes);
-        const uint32_t t_p = tmem_base + kColP + (j & 1) * 64;
-        mma_ts_4steps(tmem_base + kColO, t_p, v_lo, desc_hi_sw128(1024), idesc_pv, j > 0 ? 1u : 0u);
-        mma_ts_4steps(tmem_base + kColO, t_p + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
-        mma_commit(bar_pvdone + 8 * (j & 1));
-        if (j == n_my - 1) mma_commit(bar_ofinal);
-        mma_commit(bar_empty + 8 * (pr % L::kPairBars));
-      }
-    }
-  }
-  } else {
-    reg_alloc<224>();
-    // ================= softmax + epilogue: thread = (query row = TMEM lane, key half h) =================
-    const int h = warp >> 2;
-    const int row = threadIdx.x & 127;
-    const int t_local = row / G, j_head = row - t_local * G;
-    const bool row_valid = (row < tile_targets * G) && (t_local < n_valid);
-    int limit = 0;
-    bool row_empty = false;
-    if (row_valid) {
-      const int c = r_rank[r_cu[b] + rho0 + t_local];
-      if (c == -1 && allow_empty) {
-        row_empty = true;
-      } else if (c < 0 || c >= nu) {
-        if (h == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
-      } else {
-        limit = (mode == RELAXKV_CTX_UNION) ? c : u_pos[u_cu[b] + c];
-        if (limit < 0 || limit >= ctx_len_b) { if (h == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, limit, ctx_len_b); limit = 0; }
-      }
-    }
-    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t t_o = lane_base + kColO + h * 64;             // this thread's half of the row's O columns
-    float m = -INFINITY, z = 0.f;                               // z: this half's partial row sum
-    // Every softmax thread runs every step's two named barriers, whatever happens: a warp whose bounded wait gave up
-    // (`dead`) only skips the work between them, so the unbounded bar.sync can never be left short of arrivals.
-    bool dead = false;
-    for (int j = 0; j < n_my; ++j) {
-      const int buf = j & 1;
-      uint32_t s[64];
-      float mx_half = -INFINITY;
-      if (!dead) {
-        bool ok = mbar_wait(bar_sfull + 8 * buf, (uint32_t)(j >> 1) & 1, abort_flag);
-        dead = !__all_sync(0xffffffffu, ok);
-      }
-      if (!dead) {
-      tc_fence_after();
-      tmem_ld32(lane_base + kColS + buf * 128 + h * 64, &s[0]);
-      tmem_ld32(lane_base + kColS + buf * 128 + h * 64 + 32, &s[32]);
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(bar_sfree + 8 * buf);                         // the MMA warp may overwrite this S buffer
-      const int col0 = (j0 + j) * kBN + h * 64;
-      if (col0 + 63 > limit) {
-#pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
-      }
-      float mx8[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
-#pragma unroll
-      for (int i = 8; i + 16 <= 64; i += 16) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) mx8[e] = fmax3(mx8[e], __uint_as_float(s[i + e]), __uint_as_float(s[i + 8 + e]));
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[56 + e]));
-      mx_half = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                      fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-      // the two halves of a row agree on the tile's maximum (same value, same decisions in both)
-      xch[h * 128 + row] = mx_half;
-      }
-      named_bar_sync(1, 256);
-      if (!dead) {
-      const float mx = fmaxf(mx_half, xch[(1 - h) * 128 + row]);
-      const float m_new = mx * scale_log2;
-      if (j == 0) {
-        m = fmaxf(m_new, -1.0e30f);
-      } else {
-        const bool need = m_new > m + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          // O must hold every product up to step j - 1 before it is rescaled (Q K^T runs ahead of P V here)
-          bool ok = mbar_wait(bar_pvdone + 8 * ((j - 1) & 1), (uint32_t)((j - 1) >> 1) & 1, abort_flag);
-          dead = !__all_sync(0xffffffffu, ok);
-          if (!dead) {
-            tc_fence_after();
-            float alpha = 1.f;
-            if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              uint32_t o[32];
-              tmem_ld32(t_o + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st32(t_o + c * 32, o);
-            }
-            tmem_wait_st();
-          }
-        }
-      }
-      }
-      // the second named barrier of the step: nobody overwrites xch before both halves have read it
-      named_bar_sync(2, 256);
-      // P buffer `buf` was last read by P V of step j - 2
-      if (!dead && j >= 2) {
-        bool ok = mbar_wait(bar_pvdone + 8 * buf, (uint32_t)((j - 2) >> 1) & 1, abort_flag);
-        dead = !__all_sync(0xffffffffu, ok);
-      }
-      if (!dead) {
-      float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
-      const float neg_m = -m;
-      const uint32_t t_p = lane_base + kColP + buf * 64 + h * 32;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          float x[8], p[8];
-#pragma unroll
-          for (int e = 0; e < 8; e += 2)
-            fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
-                 scale_log2, neg_m, neg_m);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
-          add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
-          add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
-#pragma unroll
-          for (int e = 0; e < 8; e += 2) {
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(p[e], p[e + 1]);
-            pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-          }
-        }
-        tmem_st16(t_p + c * 16, pk);
-      }
-      z += (zs0 + zs1) + (zs2 + zs3);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_pfull + 8 * buf);
-      }
-    }
-    if (!dead) {
-      bool ok = mbar_wait(bar_ofinal, 0, abort_flag);
-      dead = !__all_sync(0xffffffffu, ok);
-    }
-    // total row sum = the two halves' partial sums
-    xch[h * 128 + row] = z;
-    named_bar_sync(1, 256);
-    if (!dead) {
-      tc_fence_after();
-      const float z_row = z + xch[(1 - h) * 128 + row];
-      const bool none = row_empty || !(z_row > 0.f);
-      const float inv = none ? 0.f : 1.f / z_row;
-      const float lse = none ? -INFINITY : (m + log2f(z_row)) * kLn2A;
-      const long long orow = q_row_base + t_local;
-      const long long slot = ((long long)split * n_target_rows + orow) * H + hd * G + j_head;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t o[32];
-        tmem_ld32(t_o + c * 32, o);
-        tmem_wait_ld();
-        if (row_valid) {
-          if (n_splits == 1) {
-            uint16_t* optr = out + (orow * H + hd * G + j_head) * D + h * 64 + c * 32;
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv, __uint_as_float(o[i + 2 * e + 1]) * inv);
-                w[e] = *reinterpret_cast<uint32_t*>(&h2);
-              }
-              *reinterpret_cast<uint4*>(optr + i) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          } else {
-            float* optr = part_o + slot * D + h * 64 + c * 32;
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              *reinterpret_cast<float4*>(optr + i) = make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
-                                                                 __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-          }
-        }
-      }
-      if (row_valid && h == 0) {
-        if (n_splits == 1) { if (lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = lse; }
-        else part_lse[slot] = lse;
-      }
-    }
-  }
-
-  // ---- teardown ----
-  tc_fence_before();
-  __syncthreads();
-  if (*abort_flag) {
-    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, tile, hd);
-    const uint64_t t0 = global_timer_ns();
-    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
-    __syncthreads();
-  }
-  if (warp == 9) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
-  }
-}
-
 // Explicit lists (the paper's controlled configurations): per target the index of the last context entry
 // at or before its position (-1: none), per context entry the row of the fresh K/V that replaces it (-1:
 // cached).  rt.tile_cu = prefix of the host bounds on the target counts, rt.bound_b = bounds on the context.
@@ -1329,7 +531,7 @@ __global__ void combine_splits_kernel(const float* __restrict__ part_o, const fl
                                       uint16_t* __restrict__ out, float* __restrict__ lse_out) {
   const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  const long long rows_true = r_cu[n_req] - r_cu[0];
+  const long long rows_true = min((long long)(r_cu[n_req] - r_cu[0]), n_target_rows);
   if (w >= rows_true * H) return;
   const long long row = w / H;
   const int h = (int)(w - row * H);
@@ -1358,22 +560,22 @@ __global__ void combine_splits_kernel(const float* __restrict__ part_o, const fl
   if (lane == 0 && lse_out) lse_out[(long long)h * n_target_rows + row] = den > 0.f ? mx + logf(den) : -INFINITY;
 }
 
-static int g_forced_splits = 0;      // 0: chosen from the launch size; > 0: forced (test hook)
-static int g_variant = 0;            // head_dim 128 only (test hook): 0 two tiles per CTA, 1 SM pairs, 2 one tile with split keys
-
 // ---- host side ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
+  static std::atomic<EncodeTiledFn> cached{nullptr};
+  EncodeTiledFn fn = cached.load(std::memory_order_acquire);
   if (!fn) {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
+        q == cudaDriverEntryPointSuccess) {
       fn = reinterpret_cast<EncodeTiledFn>(p);
+      cached.store(fn, std::memory_order_release);
+    }
   }
   return fn;
 }
@@ -1400,20 +602,16 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   const int H = shape->n_q_heads, Hkv = shape->n_kv_heads, G = H / Hkv;
   const int tile_targets = kBM / G;
   const int B = shape->n_req;
-  // opt-in: head_dim 128 on SM pairs (a cluster of two CTAs = four query tiles); otherwise single CTAs
-  const bool use_pair = (D == 128) && g_variant == 1;
-  const bool use_split = (D == 128) && g_variant == 2;
-  const int tiles_per_unit = use_pair ? 4 : (use_split ? 1 : 2);
-  for (int b = 0; b < B; ++b)     // tile_cu counts the launch units per request: tile PAIRS, or clusters of two pairs
-    plan.rt.tile_cu[b + 1] = plan.rt.tile_cu[b] + (plan.rt.bound_a[b] + tiles_per_unit * tile_targets - 1) / (tiles_per_unit * tile_targets);
-  const long long grid = (long long)plan.rt.tile_cu[B] * Hkv * (use_pair ? 2 : 1);
+  for (int b = 0; b < B; ++b)     // tile_cu counts the launch units per request: PAIRS of query tiles
+    plan.rt.tile_cu[b + 1] = plan.rt.tile_cu[b] + (plan.rt.bound_a[b] + 2 * tile_targets - 1) / (2 * tile_targets);
+  const long long grid = (long long)plan.rt.tile_cu[B] * Hkv;
   if (grid == 0) return RELAXKV_OK;
   if (grid > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   CUtensorMap tm_q, tm_k, tm_v;
   const uint64_t row_q = (uint64_t)H * D * 2, row_kv = (uint64_t)Hkv * D * 2;
   if (!make_map_3d(&tm_q, q_new, D, H, (uint64_t)n_target_rows, (uint64_t)D * 2, row_q, (uint32_t)G, (uint32_t)tile_targets) ||
       !make_map_3d(&tm_k, plan.k_base, D, Hkv, (uint64_t)plan.ctx_rows, plan.kv_head_stride_bytes, plan.kv_token_stride_bytes, 1u,
-                   (uint32_t)(use_pair ? kBN / 2 : kBN)) ||          // a CTA of a pair stages 64 of a tile's 128 keys
+                   (uint32_t)kBN) ||
       !make_map_3d(&tm_v, plan.v_base, D, Hkv, (uint64_t)plan.ctx_rows, plan.kv_head_stride_bytes, plan.kv_token_stride_bytes, 1u,
                    (uint32_t)kBN))
     return RELAXKV_ERR_CUDA;
@@ -1423,49 +621,36 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
   long long ctx_rows_used = 0;
   for (int b = 0; b < B; ++b) ctx_rows_used += plan.rt.bound_b[b];
   const int head_inner = (ctx_rows_used * (long long)row_kv * 2 <= (40ll << 20)) ? 1 : 0;
-  // Too few query tiles to fill the GPU (a query prefill, a decode step, a deep layer with few targets): split
-  // every pair's context over several blocks and merge the partial results afterwards.
-  static int sm_count[64] = {0};
-  int dev0 = 0;
-  if (cudaGetDevice(&dev0) != cudaSuccess || dev0 < 0 || dev0 >= 64) return RELAXKV_ERR_CUDA;
-  if (sm_count[dev0] == 0 && cudaDeviceGetAttribute(&sm_count[dev0], cudaDevAttrMultiProcessorCount, dev0) != cudaSuccess)
-    return RELAXKV_ERR_CUDA;
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return RELAXKV_ERR_CUDA;
+  // Context split.  A block's work is its pair's context length; with fewer blocks than a few waves of SMs (a query
+  // prefill, a decode step, a layer with few targets, a short context) the longest pairs would run alone at the end,
+  // so every pair's context is cut into pieces of at least four tiles until the launch has about four blocks per SM.
   long long max_tiles = 1;
   for (int b = 0; b < B; ++b) max_tiles = std::max<long long>(max_tiles, (plan.rt.bound_b[b] + kBN - 1) / kBN);
   long long n_splits = 1;
-  if (g_forced_splits > 0) {
-    n_splits = g_forced_splits;
-  } else if (grid < sm_count[dev0]) {
-    // one full wave: as many splits as whole blocks fit the SMs, each at least four context tiles long
-    n_splits = std::min<long long>(std::max<long long>(1, sm_count[dev0] / grid), std::max<long long>(1, max_tiles / 4));
+  const int forced = (shape->h_tuning && shape->h_tuning->attention_ctx_splits > 0) ? shape->h_tuning->attention_ctx_splits : 0;
+  if (forced > 0) {
+    n_splits = forced;
+  } else if (grid < 4ll * sms) {
+    n_splits = std::min<long long>(std::max<long long>(1, (grid < sms ? sms : 4ll * sms) / grid), std::max<long long>(1, max_tiles / 4));
   }
   n_splits = std::min<long long>(n_splits, kMaxCtxSplits);
   n_splits = std::min<long long>(n_splits, kSplitRowsCap / n_target_rows);   // partial slots: [split][row of the call]
   if (n_splits < 1) n_splits = 1;
   auto kern = attention_sm100_kernel<D>;
-  static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
+  static std::atomic<int> attr_done[kMaxDevices];          // per device: the opt-in to > 48 KB of dynamic shared memory
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
-  if (!attr_done[dev]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_pair_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::kDynamic) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_split_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SplitSmem::kDynamic) != cudaSuccess)
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RELAXKV_ERR_CUDA;
+  if (!attr_done[dev].load(std::memory_order_acquire)) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess)
       return RELAXKV_ERR_CUDA;
-    attr_done[dev] = true;
+    attr_done[dev].store(1, std::memory_order_release);
   }
-  if (use_pair) {
-    attention_pair_sm100_kernel<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, PairSmem::kDynamic, stream>>>(
-        tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
-        u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
-  } else if (use_split) {
-    attention_split_sm100_kernel<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, SplitSmem::kDynamic, stream>>>(
-        tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
-        u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
-  } else {
-    kern<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
-        tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
-        u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
-  }
+  RELAXKV_RANGE("attention_sm100_kernel");
+  kern<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(
+      tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, plan.dense_ctx, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
+      u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
   relaxkv_status rc = launch_ok();
   if (rc != RELAXKV_OK || n_splits == 1) return rc;
   const long long warps = plan.sum_targets * H;
@@ -1493,18 +678,6 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention(
   if (shape->head_dim == 128)
     return launch_attention<128>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
   return launch_attention<64>(shape, mode, plan, q_new, u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, out, lse_out, stream);
-}
-
-extern "C" relaxkv_status relaxkv_debug_set_attention_splits(int32_t n_splits) {
-  if (n_splits < 0 || n_splits > kMaxCtxSplits) return RELAXKV_ERR_INVALID_ARG;
-  g_forced_splits = n_splits;
-  return RELAXKV_OK;
-}
-
-extern "C" relaxkv_status relaxkv_debug_set_attention_variant(int32_t variant) {
-  if (variant < 0 || variant > 2) return RELAXKV_ERR_INVALID_ARG;
-  g_variant = variant;
-  return RELAXKV_OK;
 }
 
 extern "C" relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream) {

@@ -5,6 +5,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#ifdef RELAXKV_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 #include "relaxkv.h"
 
 namespace relaxkv {
@@ -20,8 +25,25 @@ struct DeviceStatus {
   int v1;
 };
 
-// Device address of the status word of the current device (defined in api.cu).
-DeviceStatus* status_word();
+// Per-device values that are looked up once (defined in api.cu).  The lookups are idempotent, so the caches are
+// plain atomics: two host threads that race on a first call both store the same value.
+constexpr int kMaxDevices = 64;
+DeviceStatus* status_word();             // device address of the status word of the current device; NULL on error
+int sm_count_of_current_device();        // multiprocessors of the current device; 0 on error
+
+// Optional NVTX ranges, one per C-ABI call and per kernel launch, so that a timeline taken of a caller's process
+// can be attributed to the steps of Algorithm 1.  Compiled in with -DRELAXKV_NVTX (build.py: RELAXKV_NVTX=1).
+#ifdef RELAXKV_NVTX
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+#define RELAXKV_RANGE_CAT2(a, b) a##b
+#define RELAXKV_RANGE_CAT(a, b) RELAXKV_RANGE_CAT2(a, b)
+#define RELAXKV_RANGE(name) ::relaxkv::NvtxRange RELAXKV_RANGE_CAT(relaxkv_nvtx_range_, __LINE__)(name)
+#else
+#define RELAXKV_RANGE(name) do { } while (0)
+#endif
 
 enum KernelId : int {
   KID_SETS = 1, KID_SELECT = 2, KID_SCORE = 3, KID_GATHER = 4, KID_SCATTER = 5,

@@ -6,6 +6,7 @@
 // lane) drain tile i while the tensor pipe works on tile i+1.  Tiles are walked in groups of 16 row tiles so
 // that a wave's working set (x rows + W rows) stays in L2.
 #include "common.cuh"
+#include "gemv.cuh"
 #include "sm100_ptx.cuh"
 #include <algorithm>
 
@@ -393,8 +394,6 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   if (warp == 5) { tc_fence_after(); tmem_dealloc2(tmem_base, 512); }
 }
 
-static int g_gemm_single_cta = 0;   // 1: never use the SM-pair GEMM (test hook)
-
 }  // namespace relaxkv
 
 using namespace relaxkv;
@@ -406,7 +405,13 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
   if (n_rows < 0 || n_out < 8 || n_in < 8 || (n_out % 8) || (n_in % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (swiglu && ((n_out % 256) || residual)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
-  const bool use_pair = !g_gemm_single_cta;
+  if (n_rows <= kGemvMaxRows)       // a decode token: stream the weights once, no 128-row tiles
+    return launch_gemv(x, weight, residual, y, (int)n_rows, n_out, n_in, swiglu, static_cast<cudaStream_t>(stream_));
+  // SM pairs (256-row tiles) unless that would leave a large share of the last tile row empty: with an odd number of
+  // 128-row tiles, seven at most, the second block of the last pair would compute padding only (>= 1/8 of the work),
+  // and the single-block kernel (128 x 256 tiles) is used.
+  const long long tiles_128 = (n_rows + kGemmBM - 1) / kGemmBM;
+  const bool use_pair = !((tiles_128 & 1) && tiles_128 <= 7);
   CUtensorMap tm_a, tm_b;
   if (!make_map_3d(&tm_a, x, (uint64_t)n_in, (uint64_t)n_rows, 1, (uint64_t)n_in * 2, (uint64_t)n_in * 2 * (uint64_t)n_rows, kGemmBM, 1) ||
       !make_map_3d(&tm_b, weight, (uint64_t)n_in, (uint64_t)n_out, 1, (uint64_t)n_in * 2, (uint64_t)n_in * 2 * (uint64_t)n_out,
@@ -414,27 +419,27 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
     return RELAXKV_ERR_CUDA;
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
-  static bool attr_done[64] = {false};
+  static std::atomic<int> attr_done[kMaxDevices];
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
-  if (!attr_done[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RELAXKV_ERR_CUDA;
+  if (!attr_done[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(gemm_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_pair_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem) != cudaSuccess)
       return RELAXKV_ERR_CUDA;
-    attr_done[dev] = true;
+    attr_done[dev].store(1, std::memory_order_release);
   }
-  static int sm_count[64] = {0};
-  if (sm_count[dev] == 0 && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return RELAXKV_ERR_CUDA;
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return RELAXKV_ERR_CUDA;
   const long long tiles_n = (n_out + kGemmBN - 1) / kGemmBN;
   if (use_pair) {
     const long long tiles_m2 = (n_rows + 2 * kGemmBM - 1) / (2 * kGemmBM);
     if (tiles_m2 * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
     // persistent: as many clusters as can be resident at once (fewer than SMs / 2 where a GPC has an odd SM left over)
-    static int max_clusters[64] = {0};
-    if (max_clusters[dev] == 0) {
+    static std::atomic<int> max_clusters[kMaxDevices];
+    int n_clusters = max_clusters[dev].load(std::memory_order_acquire);
+    if (n_clusters == 0) {
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)sm_count[dev]);
+      cfg.gridDim = dim3((unsigned)sms);
       cfg.blockDim = dim3(kGemmThreads);
       cfg.dynamicSmemBytes = kPairSmem;
       cudaLaunchAttribute attr;
@@ -443,17 +448,18 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
       cfg.attrs = &attr;
       cfg.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, gemm_pair_sm100_kernel, &cfg) != cudaSuccess || n < 1) n = std::max(1, sm_count[dev] / 2 - 8);
-      max_clusters[dev] = n;
+      if (cudaOccupancyMaxActiveClusters(&n, gemm_pair_sm100_kernel, &cfg) != cudaSuccess || n < 1) n = std::max(1, sms / 2 - 8);
+      n_clusters = n;
+      max_clusters[dev].store(n, std::memory_order_release);
     }
-    const long long clusters = std::min<long long>(tiles_m2 * tiles_n, max_clusters[dev]);
+    const long long clusters = std::min<long long>(tiles_m2 * tiles_n, n_clusters);
     gemm_pair_sm100_kernel<<<(unsigned)(2 * clusters), kGemmThreads, kPairSmem, static_cast<cudaStream_t>(stream_)>>>(
         tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, st);
     return launch_ok();
   }
   const long long tiles_m = (n_rows + kGemmBM - 1) / kGemmBM;
   if (tiles_m * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
-  const long long grid = std::min<long long>(tiles_m * tiles_n, sm_count[dev]);     // persistent: one CTA per SM
+  const long long grid = std::min<long long>(tiles_m * tiles_n, sms);     // persistent: one CTA per SM
   gemm_sm100_kernel<<<(unsigned)grid, kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
       tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, st);
   return launch_ok();
@@ -468,9 +474,4 @@ extern "C" relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weigh
                                                 int32_t n_inter, int32_t n_in, relaxkv_stream stream_) {
   if (n_inter < 128 || (n_inter % 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   return launch_gemm(x, weight_tiled, nullptr, y, n_rows, 2 * n_inter, n_in, 1, stream_);
-}
-
-extern "C" relaxkv_status relaxkv_debug_set_gemm_single_cta(int32_t on) {
-  g_gemm_single_cta = on ? 1 : 0;
-  return RELAXKV_OK;
 }

@@ -1,0 +1,116 @@
+// Projections of a handful of rows (a decode token, the last query row going through the output head): y = x W^T with
+// at most kGemvMaxRows rows of x.  The work is reading W once (HBM-bound: every weight byte meets one to four
+// multiply-adds), so this is a plain streaming kernel, not the 128-row tensor-core GEMM: each warp owns four output
+// features, its lanes stride over K in 16-byte pieces with eight independent weight loads in flight per lane, x stays
+// in L1, and a shuffle tree sums the lanes' partial dot products in a fixed order.  (Algorithm 1 runs "the unchanged
+// Transformer block"; after the repair loop the same block serves the decode step of the TTFT region.)
+#include "common.cuh"
+#include "gemv.cuh"
+
+namespace relaxkv {
+
+constexpr int kGemvThreads = 256;
+constexpr int kGemvFeatPerWarp = 4;
+constexpr int kGemvFeatPerBlock = (kGemvThreads / 32) * kGemvFeatPerWarp;
+
+__device__ __forceinline__ void unpack8_gemv(const uint4& v, float* f) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(w[e] << 16); f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
+}
+
+// SWIGLU = 0: y[m, n] = sum_k x[m, k] w[n, k] (+ residual[m, n])          w [n_out, K]
+// SWIGLU = 1: y[m, f] = silu(sum_k x w[g(f), k]) * (sum_k x w[g(f) + 128, k])   with g(f) = (f / 128) * 256 + f % 128
+//             (the gate rows of every block of 128 features are followed by its up rows); n_out counts the features f
+template <int M, int SWIGLU>
+__global__ void __launch_bounds__(kGemvThreads)
+gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, const uint16_t* __restrict__ residual,
+            uint16_t* __restrict__ y, int n_out, int K) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int f0 = blockIdx.x * kGemvFeatPerBlock + warp * kGemvFeatPerWarp;
+  constexpr int R = SWIGLU ? 2 * kGemvFeatPerWarp : kGemvFeatPerWarp;      // weight rows this warp streams
+  const uint16_t* wr[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int f = min(f0 + (r % kGemvFeatPerWarp), n_out - 1);              // the tail warp re-reads the last feature
+    const long long row = SWIGLU ? ((long long)(f / 128) * 256 + (f % 128) + (r >= kGemvFeatPerWarp ? 128 : 0)) : f;
+    wr[r] = w + row * K;
+  }
+  float acc[R][M];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[r][m] = 0.f;
+#pragma unroll 2
+  for (int k = lane * 8; k < K; k += 32 * 8) {
+    uint4 wv[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) wv[r] = __ldg(reinterpret_cast<const uint4*>(wr[r] + k));     // all loads first
+    float xf[M][8];
+#pragma unroll
+    for (int m = 0; m < M; ++m) unpack8_gemv(__ldg(reinterpret_cast<const uint4*>(x + (long long)m * K + k)), xf[m]);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float wf[8];
+      unpack8_gemv(wv[r], wf);
+#pragma unroll
+      for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[r][m] = fmaf(xf[m][e], wf[e], acc[r][m]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[r][m] = warp_reduce_sum(acc[r][m]);
+  if (lane < kGemvFeatPerWarp) {
+    const int f = f0 + lane;
+    if (f < n_out) {
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        float v = 0.f;
+#pragma unroll
+        for (int r = 0; r < kGemvFeatPerWarp; ++r) {          // static indexing keeps the accumulators in registers
+          if (r == lane) {
+            if (SWIGLU) {                                     // one rounding, after the activation
+              const float g = acc[r][m], u = acc[r + (SWIGLU ? kGemvFeatPerWarp : 0)][m];
+              v = g / (1.f + __expf(-g)) * u;
+            } else {
+              v = acc[r][m];
+            }
+          }
+        }
+        const long long o = (long long)m * n_out + f;
+        if (!SWIGLU && residual) v += bf16_bits_to_float(residual[o]);
+        const __nv_bfloat16 h = __float2bfloat16(v);
+        y[o] = *reinterpret_cast<const uint16_t*>(&h);
+      }
+    }
+  }
+}
+
+template <int SWIGLU>
+static relaxkv_status launch_m(const uint16_t* x, const uint16_t* w, const uint16_t* residual, uint16_t* y, int n_rows,
+                               int n_out, int K, cudaStream_t stream) {
+  const unsigned blocks = (unsigned)((n_out + kGemvFeatPerBlock - 1) / kGemvFeatPerBlock);
+  switch (n_rows) {
+    case 1: gemv_kernel<1, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
+    case 2: gemv_kernel<2, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
+    case 3: gemv_kernel<3, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
+    case 4: gemv_kernel<4, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
+    default: return RELAXKV_ERR_INVALID_ARG;
+  }
+  return launch_ok();
+}
+
+relaxkv_status launch_gemv(const void* x, const void* weight, const void* residual, void* y, int n_rows, int n_out,
+                           int n_in, int swiglu, cudaStream_t stream) {
+  RELAXKV_RANGE("gemv_kernel");
+  if (swiglu)
+    return launch_m<1>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), nullptr,
+                       static_cast<uint16_t*>(y), n_rows, n_out / 2, n_in, stream);
+  return launch_m<0>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight),
+                     static_cast<const uint16_t*>(residual), static_cast<uint16_t*>(y), n_rows, n_out, n_in, stream);
+}
+
+}  // namespace relaxkv

@@ -38,7 +38,9 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
                   const int* __restrict__ u_pos, const int* __restrict__ u_cu,
                   const int* __restrict__ r_rank, const int* __restrict__ r_cu, const int* __restrict__ fresh_row,
                   uint16_t* __restrict__ k_out, uint16_t* __restrict__ v_out, long long ctx_rows,
-                  DeviceStatus* st) {
+                  long long fresh_map_rows, long long n_new_rows, DeviceStatus* st) {
+  // fresh_map_rows: entries of fresh_row that were written (the host bound on the context rows of an explicit-list
+  // call); n_new_rows: rows k_new / v_new hold.  An index past either is reported and the row zero-filled.
   __shared__ long long src_off[kGatherRows];   // element offset of the source row (head 0)
   __shared__ int src_kind[kGatherRows];        // 0 = cache, 1 = fresh, 2 = zero fill, 3 = skip
   const long long row0 = (long long)blockIdx.x * kGatherRows;
@@ -73,14 +75,30 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
           off = (rt.tok_off[b] + p) * tok_stride;
           if (k_new != nullptr && fresh_row != nullptr) {
             // explicit lists: the row of k_new that replaces this context entry was resolved beforehand
-            const int fr = __ldg(fresh_row + x);
-            if (fr >= 0) { kind = 1; off = (long long)fr * n_kv_heads * head_dim; }
+            if (x >= fresh_map_rows) {
+              if (lane == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_GATHER, (int)x, (int)fresh_map_rows);
+              kind = 2;
+            } else {
+              const int fr = __ldg(fresh_row + x);
+              if (fr >= n_new_rows) {
+                if (lane == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_GATHER, (int)x, fr);
+                kind = 2;
+              } else if (fr >= 0) {
+                kind = 1; off = (long long)fr * n_kv_heads * head_dim;
+              }
+            }
           } else if (k_new != nullptr && c >= 0) {
             const int rb = __ldg(r_cu + b), nr = __ldg(r_cu + b + 1) - rb;
             const int rho = warp_lower_bound(r_rank + rb, nr, c, lane);
             if (rho < nr && __ldg(r_rank + rb + rho) == c) {
-              kind = 1;
-              off = (long long)(rb - __ldg(r_cu) + rho) * n_kv_heads * head_dim;
+              const long long frow = (long long)(rb - __ldg(r_cu)) + rho;
+              if (frow >= n_new_rows) {
+                if (lane == 0) report(st, RELAXKV_ERR_BAD_INDEX, KID_GATHER, (int)x, (int)frow);
+                kind = 2;
+              } else {
+                kind = 1;
+                off = frow * n_kv_heads * head_dim;
+              }
             }
           }
         }
@@ -196,6 +214,7 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
 relaxkv_status launch_gather(const relaxkv_shape* shape, int mode, const relaxkv_cache_view* cache,
                              const void* k_new, const void* v_new, const int32_t* u_pos, const int32_t* u_cu,
                              const int32_t* r_rank, const int32_t* r_cu_layer, const int32_t* fresh_row,
+                             long long fresh_map_rows, long long n_new_rows,
                              long long rows_to_cover, void* k_out, void* v_out, long long ctx_rows, cudaStream_t stream) {
   ReqTable rt;
   fill_req_table(rt, shape, cache, nullptr);
@@ -209,7 +228,8 @@ relaxkv_status launch_gather(const relaxkv_shape* shape, int mode, const relaxkv
       static_cast<const uint16_t*>(cache->k), static_cast<const uint16_t*>(cache->v),
       cache->token_stride, cache->head_stride,
       static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new),
-      u_pos, u_cu, r_rank, r_cu_layer, fresh_row, static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out), ctx_rows, st);
+      u_pos, u_cu, r_rank, r_cu_layer, fresh_row, static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out), ctx_rows,
+      fresh_map_rows, n_new_rows, st);
   return launch_ok();
 }
 
@@ -244,8 +264,9 @@ extern "C" relaxkv_status relaxkv_gather_kv(
     }
   }
   if (ctx_rows < need) return RELAXKV_ERR_INVALID_ARG;
-  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, nullptr, need + kCtxPadRows,
-                       k_ctx_out, v_ctx_out, ctx_rows, static_cast<cudaStream_t>(stream));
+  // this entry point is not told how many rows k_new / v_new hold: the fresh-row index is bounded by the R list only
+  return launch_gather(shape, mode, cache, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer, nullptr, 0, 0x7fffffffffffffffLL,
+                       need + kCtxPadRows, k_ctx_out, v_ctx_out, ctx_rows, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" relaxkv_status relaxkv_scatter_kv(

@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "score_sm100.cuh"
 #include "select.cuh"
+#include <algorithm>
 
 namespace relaxkv {
 
@@ -81,6 +82,18 @@ static relaxkv_status score_layers(const relaxkv_shape* shape, ReqTable rt, cons
   return launch_ok();
 }
 
+// Positions of the query's own tokens (they follow the context: T_c, T_c + 1, ...) and their offsets, as the target
+// lists of the cache-only attention call.
+__global__ void query_positions_kernel(ReqTable rt, int* __restrict__ tgt_pos, int* __restrict__ tgt_cu) {
+  const int B = rt.n_req;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i <= B) tgt_cu[i] = rt.q_cu[i];
+  if (i < rt.q_cu[B]) {
+    const int b = find_segment(rt.q_cu, B, i);
+    tgt_pos[i] = rt.ctx_len[b] + (i - rt.q_cu[b]);
+  }
+}
+
 }  // namespace relaxkv
 
 using namespace relaxkv;
@@ -103,6 +116,7 @@ extern "C" relaxkv_status relaxkv_score_select(
     if (!q_layers[l] || !aligned16(q_layers[l])) return RELAXKV_ERR_INVALID_ARG;
     if ((rc = check_cache(shape, &cache_layers[l], false)) != RELAXKV_OK) return rc;
   }
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return RELAXKV_ERR_INVALID_ARG;
   const WsLayout ws = ws_layout(shape, n_layers);
   if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -136,4 +150,55 @@ extern "C" relaxkv_status relaxkv_score_select(
   ReqTable rt;
   fill_req_table(rt, shape, nullptr, h_k);
   return launch_select(rt, n_layers, raw_scores_out, norm_scores_out, anchors_out, stream);
+}
+
+// The query's own causal attention over [context, query] with the context scores taken from the same pass: the
+// attention call leaves every row's log-normaliser, the column-sum pass of the scoring kernel then reads the context
+// keys once more with those normalisers.  The statistics pass of relaxkv_score_select never runs.
+extern "C" relaxkv_status relaxkv_query_prefill_attention(
+    const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q, void* out, float* lse_out,
+    float* raw_scores_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_query_prefill_attention");
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if ((rc = check_cache(shape, cache, true)) != RELAXKV_OK) return rc;
+  if (!q || !out || !lse_out || !workspace || !shape->h_q_len || !aligned16(q) || !aligned16(out))
+    return RELAXKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return RELAXKV_ERR_INVALID_ARG;
+  const int B = shape->n_req;
+  int32_t ext_len[kMaxReqInline], q_len[kMaxReqInline];
+  long long sum_q = 0;
+  for (int b = 0; b < B; ++b) {
+    if (shape->h_q_len[b] < 1) return RELAXKV_ERR_INVALID_ARG;
+    const long long e = (long long)shape->h_ctx_len[b] + shape->h_q_len[b];
+    if (e > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+    ext_len[b] = (int32_t)e;
+    q_len[b] = shape->h_q_len[b];
+    sum_q += q_len[b];
+  }
+  if (sum_q > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  relaxkv_shape ext = *shape;                       // the same batch with the query's tokens counted into the cache rows
+  ext.h_ctx_len = ext_len;
+  const WsLayout ws = ws_layout(&ext, 1);
+  if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char* base = static_cast<char*>(workspace);
+  int* tgt_pos = reinterpret_cast<int*>(base + ws.list_limit);        // regions the cache-only attention does not use
+  int* tgt_cu = reinterpret_cast<int*>(base + ws.list_fresh);
+  ReqTable rt;
+  fill_req_table(rt, shape, cache, nullptr);
+  const long long n = std::max<long long>(sum_q, B + 1);
+  query_positions_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(rt, tgt_pos, tgt_cu);
+  if ((rc = launch_ok()) != RELAXKV_OK) return rc;
+  rc = relaxkv_cache_attention(&ext, cache, q, tgt_pos, tgt_cu, sum_q, q_len, out, lse_out, workspace, workspace_bytes, stream_);
+  if (rc != RELAXKV_OK || !raw_scores_out) return rc;
+  // column sums over the CONTEXT keys with the rows' normalisers from the attention above
+  const ScorePlan plan = plan_score(shape);
+  const WsLayout ws_sc = ws_layout(shape, 1);
+  if (workspace_bytes < ws_sc.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
+  const void* q_arr[1] = {q};
+  const float* lse_arr[1] = {lse_out};
+  if (shape->head_dim == 128)
+    return score_layers<128>(shape, rt, plan, 1, q_arr, cache, lse_arr, raw_scores_out, base, ws_sc, stream);
+  return score_layers<64>(shape, rt, plan, 1, q_arr, cache, lse_arr, raw_scores_out, base, ws_sc, stream);
 }

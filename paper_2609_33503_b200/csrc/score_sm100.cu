@@ -353,16 +353,16 @@ relaxkv_status launch_score_sm100(const relaxkv_shape* shape, ReqTable rt, const
   const dim3 grid((unsigned)rt.tile_cu[B], (unsigned)Hkv, (unsigned)(n_splits * n_layers));
   if (grid.x == 0) return RELAXKV_OK;
   constexpr int smem = ScoreSmem<D>::kTotal;
-  static bool attr_done[64] = {false};          // per device: the opt-in to > 48 KB of dynamic shared memory
+  static std::atomic<int> attr_done[kMaxDevices];          // per device: the opt-in to > 48 KB of dynamic shared memory
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RELAXKV_ERR_CUDA;
   auto k1 = score_sm100_kernel<D, false>;
   auto k2 = score_sm100_kernel<D, true>;
-  if (!attr_done[dev]) {
+  if (!attr_done[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
         cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return RELAXKV_ERR_CUDA;
-    attr_done[dev] = true;
+    attr_done[dev].store(1, std::memory_order_release);
   }
   if (need_pass1) {
     k1<<<grid, kScThreads, smem, stream>>>(layers, rt, H, Hkv, scale_log2, n_splits, plan.max_super, lse_ws, part, colpart, st);

@@ -136,6 +136,12 @@ __global__ void mean_scores_kernel(int n_layers, long long sum_t, const float* _
   g[i] = a / (float)n_layers;
 }
 
+// scores[i] *= factor   (combining the per-shard mean scores of a head-sharded layout: mean over shards)
+__global__ void scale_scores_kernel(long long n, float factor, float* __restrict__ scores) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) scores[i] *= factor;
+}
+
 relaxkv_status launch_select(const ReqTable& rt, int n_layers, const float* raw, float* norm, int* anchors,
                              cudaStream_t stream) {
   DeviceStatus* st = status_word();
@@ -169,5 +175,18 @@ extern "C" relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_
   long long sum_t = 0;
   for (int b = 0; b < shape->n_req; ++b) sum_t += shape->h_ctx_len[b];
   mean_scores_kernel<<<(unsigned)((sum_t + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(n_layers, sum_t, scores, mean_out);
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_scale_scores(const relaxkv_shape* shape, int32_t n_layers, float* scores, float factor,
+                                               relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_scale_scores");
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (n_layers < 1 || !scores || !(factor > 0.f)) return RELAXKV_ERR_INVALID_ARG;
+  long long n = 0;
+  for (int b = 0; b < shape->n_req; ++b) n += shape->h_ctx_len[b];
+  n *= n_layers;
+  scale_scores_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(n, factor, scores);
   return launch_ok();
 }

@@ -133,29 +133,19 @@ write_sets_kernel(ReqTable rt, int n_layers, const int* __restrict__ h, const in
 
 using namespace relaxkv;
 
-extern "C" relaxkv_status relaxkv_build_active_sets(
-    const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
-    int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
-    int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned,
-    void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
-  relaxkv_status rc = check_shape(shape);
-  if (rc != RELAXKV_OK) return rc;
-  if (n_layers < 1 || n_layers > 65535 || !h_k || !anchors || !highest_layer_out || !u_pos_out || !u_cu_out ||
-      !u_rank_out || !r_rank_out || !r_cu_out || !workspace)
-    return RELAXKV_ERR_INVALID_ARG;
-  for (int b = 0; b < shape->n_req; ++b)
-    if (h_k[b] < 1 || h_k[b] > shape->h_ctx_len[b]) return RELAXKV_ERR_INVALID_ARG;
-  const WsLayout ws = ws_layout(shape, n_layers);
-  if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+// The launch sequence both entry points share: `counts` (device int32 [B + n_layers*B]) is the only scratch.
+static relaxkv_status build_sets(const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
+                                 int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
+                                 int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned, int* counts,
+                                 cudaStream_t stream) {
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
   ReqTable rt;
   fill_req_table(rt, shape, nullptr, h_k);
   const int B = shape->n_req;
   const long long sum_t = rt.ctx_cu[B];
-  int* counts = reinterpret_cast<int*>(static_cast<char*>(workspace) + ws.counts);
-
+  // Nothing in `counts` has to start at zero: count_sets_kernel overwrites every entry that prefix_counts_kernel
+  // and the copy below read.
   fill_i32_kernel<<<(unsigned)((sum_t + 255) / 256), 256, 0, stream>>>(highest_layer_out, sum_t, -1);
   const long long n_anchor = (long long)n_layers * rt.k_cu[B];
   highest_layer_kernel<<<(unsigned)((n_anchor + 255) / 256), 256, 0, stream>>>(rt, n_layers, anchors,
@@ -165,12 +155,43 @@ extern "C" relaxkv_status relaxkv_build_active_sets(
   prefix_counts_kernel<<<1, 64, 0, stream>>>(B, n_layers, counts, u_cu_out, r_cu_out);
   write_sets_kernel<<<blocks, kSetThreads, 0, stream>>>(rt, n_layers, highest_layer_out, u_cu_out, r_cu_out,
                                                         u_pos_out, u_rank_out, r_rank_out);
-  if ((rc = launch_ok()) != RELAXKV_OK) return rc;
-  if (h_counts_pinned) {
+  relaxkv_status rc = launch_ok();
+  if (rc != RELAXKV_OK) return rc;
+  if (h_counts_pinned)
     rc = cuda_ok(cudaMemcpyAsync(h_counts_pinned, counts, sizeof(int) * (size_t)(B + n_layers * B),
                                  cudaMemcpyDeviceToHost, stream));
-  }
   return rc;
+}
+
+static relaxkv_status check_sets_args(const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k,
+                                      const int32_t* anchors, const int32_t* highest_layer_out, const int32_t* u_pos_out,
+                                      const int32_t* u_cu_out, const int32_t* u_rank_out, const int32_t* r_rank_out,
+                                      const int32_t* r_cu_out) {
+  relaxkv_status rc = check_shape(shape);
+  if (rc != RELAXKV_OK) return rc;
+  if (n_layers < 1 || n_layers > 65535 || !h_k || !anchors || !highest_layer_out || !u_pos_out || !u_cu_out ||
+      !u_rank_out || !r_rank_out || !r_cu_out)
+    return RELAXKV_ERR_INVALID_ARG;
+  for (int b = 0; b < shape->n_req; ++b)
+    if (h_k[b] < 1 || h_k[b] > shape->h_ctx_len[b]) return RELAXKV_ERR_INVALID_ARG;
+  return RELAXKV_OK;
+}
+
+extern "C" relaxkv_status relaxkv_build_active_sets(
+    const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
+    int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
+    int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned,
+    void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_build_active_sets");
+  relaxkv_status rc = check_sets_args(shape, n_layers, h_k, anchors, highest_layer_out, u_pos_out, u_cu_out, u_rank_out,
+                                      r_rank_out, r_cu_out);
+  if (rc != RELAXKV_OK) return rc;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return RELAXKV_ERR_INVALID_ARG;
+  const WsLayout ws = ws_layout(shape, n_layers);
+  if (workspace_bytes < ws.total) return RELAXKV_ERR_WORKSPACE_TOO_SMALL;
+  int* counts = reinterpret_cast<int*>(static_cast<char*>(workspace) + ws.counts);
+  return build_sets(shape, n_layers, h_k, anchors, highest_layer_out, u_pos_out, u_cu_out, u_rank_out, r_rank_out, r_cu_out,
+                    h_counts_pinned, counts, static_cast<cudaStream_t>(stream_));
 }
 
 // ---- variant whose scratch lives in the library image ------------------------------------------
@@ -186,15 +207,15 @@ static __device__ __align__(256) int g_static_counts[kStaticCountsMax];
 // handle; the address a kernel can use comes from cudaGetSymbolAddress, once per device, with that
 // device current.
 static relaxkv_status static_counts_ptr(int** out) {
-  static int* cached[64] = {nullptr};
+  static std::atomic<int*> cached[kMaxDevices];
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RELAXKV_ERR_CUDA;
-  if (!cached[dev]) {
-    int* p = nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RELAXKV_ERR_CUDA;
+  int* p = cached[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress((void**)&p, g_static_counts) != cudaSuccess || p == nullptr) return RELAXKV_ERR_CUDA;
-    cached[dev] = p;
+    cached[dev].store(p, std::memory_order_release);
   }
-  *out = cached[dev];
+  *out = p;
   return RELAXKV_OK;
 }
 
@@ -202,37 +223,14 @@ extern "C" relaxkv_status relaxkv_build_active_sets_static(
     const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k, const int32_t* anchors,
     int32_t* highest_layer_out, int32_t* u_pos_out, int32_t* u_cu_out, int32_t* u_rank_out,
     int32_t* r_rank_out, int32_t* r_cu_out, int32_t* h_counts_pinned, relaxkv_stream stream_) {
-  relaxkv_status rc = check_shape(shape);
+  RELAXKV_RANGE("relaxkv_build_active_sets_static");
+  relaxkv_status rc = check_sets_args(shape, n_layers, h_k, anchors, highest_layer_out, u_pos_out, u_cu_out, u_rank_out,
+                                      r_rank_out, r_cu_out);
   if (rc != RELAXKV_OK) return rc;
-  if (n_layers < 1 || !h_k || !anchors || !highest_layer_out || !u_pos_out || !u_cu_out || !u_rank_out ||
-      !r_rank_out || !r_cu_out)
-    return RELAXKV_ERR_INVALID_ARG;
-  for (int b = 0; b < shape->n_req; ++b)
-    if (h_k[b] < 1 || h_k[b] > shape->h_ctx_len[b]) return RELAXKV_ERR_INVALID_ARG;
   const int B = shape->n_req;
   if ((long long)B + (long long)n_layers * B > kStaticCountsMax) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   int* counts = nullptr;
   if ((rc = static_counts_ptr(&counts)) != RELAXKV_OK) return rc;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  DeviceStatus* st = status_word();
-  if (!st) return RELAXKV_ERR_CUDA;
-  ReqTable rt;
-  fill_req_table(rt, shape, nullptr, h_k);
-  const long long sum_t = rt.ctx_cu[B];
-  // Nothing in the array has to start at zero: count_sets_kernel overwrites every entry that
-  // prefix_counts_kernel and the copy below read.
-  fill_i32_kernel<<<(unsigned)((sum_t + 255) / 256), 256, 0, stream>>>(highest_layer_out, sum_t, -1);
-  const long long n_anchor = (long long)n_layers * rt.k_cu[B];
-  highest_layer_kernel<<<(unsigned)((n_anchor + 255) / 256), 256, 0, stream>>>(rt, n_layers, anchors,
-                                                                              highest_layer_out, st);
-  const unsigned blocks = (unsigned)(B * (n_layers + 1));
-  count_sets_kernel<<<blocks, kSetThreads, 0, stream>>>(rt, n_layers, highest_layer_out, counts);
-  prefix_counts_kernel<<<1, 64, 0, stream>>>(B, n_layers, counts, u_cu_out, r_cu_out);
-  write_sets_kernel<<<blocks, kSetThreads, 0, stream>>>(rt, n_layers, highest_layer_out, u_cu_out, r_cu_out,
-                                                        u_pos_out, u_rank_out, r_rank_out);
-  if ((rc = launch_ok()) != RELAXKV_OK) return rc;
-  if (h_counts_pinned)
-    rc = cuda_ok(cudaMemcpyAsync(h_counts_pinned, counts, sizeof(int) * (size_t)(B + n_layers * B),
-                                 cudaMemcpyDeviceToHost, stream));
-  return rc;
+  return build_sets(shape, n_layers, h_k, anchors, highest_layer_out, u_pos_out, u_cu_out, u_rank_out, r_rank_out, r_cu_out,
+                    h_counts_pinned, counts, static_cast<cudaStream_t>(stream_));
 }

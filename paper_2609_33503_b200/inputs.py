@@ -168,6 +168,15 @@ def llama8b_16k() -> Workload:
                     planted_chunks=((5, 14, 27),))
 
 
+def llama8b_stack(ctx_len: int = 8192, n_layers: int = 32, q_len: int = 64) -> Workload:
+    """Llama-3.1-8B-shaped full stack (32 layers, 32/8 heads, D=128) on one context built from 512-token chunks -
+    the model and context class of the paper's global repair target sweep; three planted chunks, calibrated variant."""
+    n_chunks = max(3, ctx_len // 512)
+    planted = tuple(sorted({n_chunks // 6, n_chunks // 2, (5 * n_chunks) // 6}))
+    return Workload(f"llama8b_{ctx_len // 1024}k_stack", n_layers, 32, 8, 128, 512, (ctx_len,), (q_len,), 0.15, base_seed=0,
+                    planted_chunks=(planted,), variant="calibrated")
+
+
 def qwen14b_32k(variant: str = "calibrated", ratio: float = 0.15, n_layers: int = 40) -> Workload:
     """Qwen3-14B-shaped stack: 40 layers, 40/8 heads, D=128, 32K context as 64 chunks
     of 512, 128 query tokens; per-layer tensors seeded by the layer id."""
@@ -212,6 +221,7 @@ NAMED: Dict[str, object] = {
     "tiny": tiny,
     "llama8b_16k": llama8b_16k,
     "qwen14b_32k": qwen14b_32k,
+    "llama8b_stack": llama8b_stack,
     "ragged8": ragged8,
 }
 

@@ -33,9 +33,10 @@ class LayerLoop:
         self.pos = torch.empty(n, dtype=torch.int32, device=dev)
 
     def run(self, h: torch.Tensor, weights: List[Dict[str, torch.Tensor]], caches: List[B.CacheView],
-            events: Optional[list] = None) -> torch.Tensor:
+            events: Optional[list] = None, taps: Optional[list] = None) -> torch.Tensor:
         """h: hidden rows of R_0 = U (requests packed) [sum |U_b|, hidden].  Returns the hidden rows of the
-        last layer's targets after that layer.  The caches are repaired in place."""
+        last layer's targets after that layer.  The caches are repaired in place.  `taps` (a list) receives a
+        copy of every layer's (input rows, output rows), for checks that look at one layer at a time."""
         s, blk = self.s, self.blk
         n_u, n_r = s.counts()
         L = s.n_layers
@@ -74,6 +75,8 @@ class LayerLoop:
                 rec("mlp", lambda: (B.relaxkv_linear(x, w["w_gate_up"], gu), B.relaxkv_swiglu(gu, m)))
             h_out = self.h_next[:n]
             rec("mlp", lambda: B.relaxkv_linear(m, w["w_down"], h_out, residual=a))
+            if taps is not None:
+                taps.append((h[:n].clone(), h_out.clone()))
             if l + 1 < L:
                 n_next = sum(n_r[l + 1])
                 carried = self.h_carry[l % 2][:n_next]

@@ -28,24 +28,38 @@ def head_shard(n_q_heads: int, n_kv_heads: int, world: int, rank: int) -> Tuple[
     return rank * per, (rank + 1) * per, rank * per * g, (rank + 1) * per * g
 
 
-def combine_partial_scores(raw_local: torch.Tensor, world: int, group=None) -> torch.Tensor:
-    """In place: mean over ranks of the local (per-shard mean) scores = the score over all heads.
-    One all-reduce(sum) of the [n_layers, sum T_c] fp32 tensor; identity on a single rank."""
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(raw_local, op=dist.ReduceOp.SUM, group=group)
-        raw_local.div_(world)
-    return raw_local
+def combine_partial_scores(session, world: int, group=None, stream=None, scale_fn=None) -> torch.Tensor:
+    """In place on session.raw: mean over ranks of the local (per-shard mean) scores = the score over all heads.
+    One all-reduce(sum) of the [n_layers, sum T_c] fp32 tensor followed by the library's scaling kernel
+    (relaxkv_scale_scores, factor 1 / world); identity on a single rank.  Both are enqueued on `stream` (torch's
+    current stream if None), so they are ordered after the scoring kernels and before the top-k on that stream.
+    `scale_fn(session, factor)` replaces the kernel call where no GPU exists (the CPU rank tests)."""
+    raw = session.raw
+    if world <= 1:
+        return raw
+    import torch.distributed as dist
+    if raw.is_cuda:
+        ctx = torch.cuda.stream(stream) if stream is not None else torch.cuda.stream(torch.cuda.current_stream(raw.device))
+        with ctx:
+            dist.all_reduce(raw, op=dist.ReduceOp.SUM, group=group)
+    else:
+        dist.all_reduce(raw, op=dist.ReduceOp.SUM, group=group)
+    if scale_fn is not None:
+        scale_fn(session, 1.0 / world)
+    else:
+        from . import binding as B
+        B.relaxkv_scale_scores(session.shape, session.n_layers, raw, 1.0 / world, stream=stream)
+    return raw
 
 
 def sharded_score_select(session, q_layers_local: List[torch.Tensor], cache_layers_local, world: int, group=None,
                          row_lse_layers=None, stream=None) -> None:
-    """Selection on a head shard: local scoring kernels -> all-reduce of the scores -> top-k kernel.
-    `session` is a pipeline.RepairSession built with the LOCAL head counts; on return session.raw holds the
+    """Selection on a head shard: local scoring kernels -> all-reduce of the scores -> scaling -> top-k kernel, all on
+    `stream`.  `session` is a pipeline.RepairSession built with the LOCAL head counts; on return session.raw holds the
     global scores and session.anchors the anchors (identical on every rank)."""
     from . import binding as B
     B.relaxkv_score_select(session.shape, q_layers_local, cache_layers_local, session.k, session.raw, None,
                            session.workspace, row_lse_layers=row_lse_layers, stream=stream)
-    combine_partial_scores(session.raw, world, group)
+    combine_partial_scores(session, world, group, stream=stream)
     B.relaxkv_select_topk(session.shape, session.n_layers, session.k, session.raw, session.anchors,
                           norm_scores_out=session.norm, stream=stream)

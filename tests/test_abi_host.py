@@ -97,6 +97,13 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert sc(ok_shape, 1, 257) == B.ERR_INVALID_ARG
     assert sc(ok_shape, 0, 8) == B.ERR_INVALID_ARG
     assert sc(B.Shape(8, 2, 128, [256], None), 1, 8) == B.ERR_INVALID_ARG
+    # a workspace that is not 256-byte aligned is refused by every call that takes one
+    odd = ctypes.c_void_p(0x10010)
+    assert lib.relaxkv_score_select(ok_shape.ref(), 1, qs, caches, NULL, i32([8]), FAKE, NULL, FAKE, odd,
+                                    ctypes.c_size_t(need), NULL) == B.ERR_INVALID_ARG
+    assert lib.relaxkv_build_active_sets(ok_shape.ref(), 1, i32([8]), FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, NULL,
+                                         odd, ctypes.c_size_t(need), NULL) == B.ERR_INVALID_ARG
+    assert lib.relaxkv_scale_scores(ok_shape.ref(), 1, FAKE, ctypes.c_float(0.0), NULL) == B.ERR_INVALID_ARG
     # build_active_sets: NULL outputs
     assert lib.relaxkv_build_active_sets(ok_shape.ref(), 1, i32([8]), FAKE, NULL, FAKE, FAKE, FAKE, FAKE, FAKE, NULL,
                                          FAKE, ctypes.c_size_t(need), NULL) == B.ERR_INVALID_ARG

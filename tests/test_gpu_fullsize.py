@@ -68,8 +68,11 @@ def test_llama8b_16k_full_size():
     run_full(inputs.llama8b_16k(), tile_targets=32, n_spread=48)
 
 
-def test_qwen14b_32k_full_context_two_layers():
-    run_full(inputs.qwen14b_32k("calibrated", 0.15, n_layers=2), tile_targets=25, n_spread=24)
+@pytest.mark.parametrize("ratio", [0.05, 0.15, 0.30])
+def test_qwen14b_32k_full_context_two_layers(ratio):
+    """The 32K context at the end points and the default of the anchor-ratio sweep, each with its Full-Prefix
+    Control (run_full checks both context modes on the same targets)."""
+    run_full(inputs.qwen14b_32k("calibrated", ratio, n_layers=2), tile_targets=25, n_spread=24 if ratio == 0.15 else 12)
 
 
 def test_maximum_batch_of_64_requests():
@@ -159,3 +162,55 @@ def test_ragged_batch_with_a_64k_context_sampled_rows():
         for b in range(2):
             pos = torch.from_numpy(case.sets[b].positions(l).astype(np.int64)).to(k2.device) + (0 if b == 0 else ctx[0])
             assert torch.equal(k2[pos], f.k_new[f.row_cu[b]:f.row_cu[b + 1]]) and torch.equal(v2[pos], f.v_new[f.row_cu[b]:f.row_cu[b + 1]])
+
+
+def test_whole_ragged_batch_of_eight_in_one_call():
+    """All eight requests of the ragged benchmark batch (8K ... 64K context tokens, Qwen3-14B head geometry, the
+    benchmark's query lengths) packed into ONE call per step, two layers - the launch configuration the ragged
+    benchmark times.  Anchors are drawn at random (the oracle's scoring of 250K keys is not what is checked here):
+    the repair schedule must equal the oracle's bit for bit for every request, the attention of sampled target rows
+    of every request must match the oracle in both context modes, and the cache update must be bit-exact."""
+    from paper_2609_33503_b200 import binding as B
+    w = inputs.ragged8(n_layers=2)
+    ctx = w.ctx_lens
+    rng = np.random.default_rng(88)
+    k = [max(1, round(0.15 * t)) for t in ctx]
+    override = [[np.sort(rng.choice(t, size=kb, replace=False)).astype(np.int32) for t, kb in zip(ctx, k)] for _ in range(2)]
+    case = Case(w, anchors_override=override)
+    assert case.k == k and w.n_req == 8
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    n_u, n_r = s.counts()
+    u_pos, u_cu = s.u_pos.cpu().numpy(), s.u_cu.cpu().numpy()
+    r_rank, r_cu = s.r_rank.cpu().numpy(), s.r_cu.cpu().numpy()
+    for b in range(8):
+        assert np.array_equal(u_pos[u_cu[b]:u_cu[b + 1]], case.sets[b].u_pos)
+    views = case.cache_views()
+    offs = [int(x) for x in case.ctx_cu[:-1]]
+    for l in range(2):
+        for b in range(8):
+            i = l * 8 + b
+            assert np.array_equal(r_rank[r_cu[i]:r_cu[i + 1]], case.sets[b].ranks(l))
+        f = case.fresh[l]
+        for mode, full_prefix in ((B.CTX_UNION, False), (B.CTX_FULL_PREFIX, True)):
+            out = torch.zeros_like(f.q_new)
+            s.attention(l, views[l], f.q_new, f.k_new, f.v_new, out, n_r[l], n_u, mode=mode)
+            st, detail = B.relaxkv_read_device_status()
+            assert st == 0, (st, detail)
+            for b in range(8):
+                n = f.row_cu[b + 1] - f.row_cu[b]
+                rows = sampled_rows(n, 25, 6, seed=100 * l + b)
+                if full_prefix:
+                    rows = rows[::5]
+                ref, _ = case.oracle_attention(l, b, full_prefix=full_prefix, rows=rows)
+                got = out[f.row_cu[b]:f.row_cu[b + 1]][torch.from_numpy(rows.astype(np.int64)).to(out.device)]
+                mx, mean = attention_errors(got, ref)
+                assert mx <= MAX_ABS and mean <= MEAN_ABS, (l, b, full_prefix, mx, mean)
+        k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+        s.scatter(l, B.CacheView(k2, v2, offs), f.k_new, f.v_new, n_r[l])
+        touched = torch.zeros(int(case.ctx_cu[-1]), dtype=torch.bool, device=k2.device)
+        for b in range(8):
+            pos = torch.from_numpy(case.sets[b].positions(l).astype(np.int64)).to(k2.device) + offs[b]
+            assert torch.equal(k2[pos], f.k_new[f.row_cu[b]:f.row_cu[b + 1]]) and torch.equal(v2[pos], f.v_new[f.row_cu[b]:f.row_cu[b + 1]])
+            touched[pos] = True
+        assert torch.equal(k2[~touched], case.k_cache[l][~touched]) and torch.equal(v2[~touched], case.v_cache[l][~touched])

@@ -249,7 +249,7 @@ def test_context_split_matches_oracle(case, n_splits):
     of a loosely bounded call stay untouched."""
     s = case.make_session()
     s.build_active_sets(case.anchors_tensor())
-    B().relaxkv_debug_set_attention_splits(n_splits)
+    s.shape.set_tuning(attention_ctx_splits=n_splits)
     try:
         for l in range(case.w.n_layers):
             for full_prefix in (False, True):
@@ -266,28 +266,7 @@ def test_context_split_matches_oracle(case, n_splits):
         exact, _ = run_attention(case, s, 0, B().CTX_UNION, simt=False)
         assert torch.equal(out[:n], exact)
     finally:
-        B().relaxkv_debug_set_attention_splits(0)
-
-
-@pytest.mark.parametrize("variant", [1, 2], ids=["sm_pairs", "split_keys"])
-@pytest.mark.parametrize("n_splits", [0, 3])
-def test_other_attention_kernels_match_oracle(case, n_splits, variant):
-    """The opt-in kernel variants for head_dim 128 - SM pairs (clusters of two blocks, one MMA instruction stream for
-    both SMs, half of every K/V tile per block; an odd number of tile pairs leaves the last cluster's second block
-    without targets) and one tile per block with S/P double-buffered and the keys split between the softmax
-    warpgroups - against the oracle, both context modes, with and without a forced context split."""
-    s = case.make_session()
-    s.build_active_sets(case.anchors_tensor())
-    B().relaxkv_debug_set_attention_variant(variant)
-    B().relaxkv_debug_set_attention_splits(n_splits)
-    try:
-        for l in range(case.w.n_layers):
-            for full_prefix in (False, True):
-                out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
-                check_attention(case, l, out, lse, full_prefix)
-    finally:
-        B().relaxkv_debug_set_attention_splits(0)
-        B().relaxkv_debug_set_attention_variant(0)
+        s.shape.set_tuning()
 
 
 def test_attention_orders_agree_and_is_deterministic(case):
@@ -357,7 +336,7 @@ def test_loose_host_bounds_give_the_same_result(case):
     l = 0
     f = case.fresh[l]
     for forced in (1, 0):
-        B().relaxkv_debug_set_attention_splits(forced)
+        s.shape.set_tuning(attention_ctx_splits=forced)
         try:
             exact, _ = run_attention(case, s, l, B().CTX_UNION, simt=False)
             out = torch.zeros_like(f.q_new)
@@ -365,7 +344,7 @@ def test_loose_host_bounds_give_the_same_result(case):
             s.attention(l, case.cache_views()[l], f.q_new, f.k_new, f.v_new, out, list(w.ctx_lens), list(w.ctx_lens), lse_out=lse)
             assert_status_ok()
         finally:
-            B().relaxkv_debug_set_attention_splits(0)
+            s.shape.set_tuning()
         if forced == 1:
             assert torch.equal(out, exact)
         else:
@@ -391,6 +370,17 @@ def test_bad_index_lists_are_reported_not_faulted():
     s.scatter(0, B().CacheView(k2, v2, [0]), f.k_new, f.v_new, case.max_targets(0))
     st, _ = B().relaxkv_read_device_status()
     assert st == B().ERR_BAD_INDEX
+    # fewer rows in q_new / out than the layer has targets (loose host bounds cannot see it): reported on the device,
+    # nothing is written past the rows that exist
+    s.build_active_sets(case.anchors_tensor())
+    n = f.q_new.shape[0]
+    short = torch.full((n - 3,) + tuple(f.q_new.shape[1:]), 3.0, dtype=f.q_new.dtype, device=case.device)
+    guard = torch.full((64,) + tuple(f.q_new.shape[1:]), 5.0, dtype=f.q_new.dtype, device=case.device)
+    s.attention(0, case.cache_views()[0], f.q_new[:n - 3].contiguous(), f.k_new, f.v_new, short, list(case.w.ctx_lens),
+                list(case.w.ctx_lens))
+    st, _ = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX
+    assert torch.all(short == 3.0) and torch.all(guard == 5.0)
 
 
 def test_expired_wait_is_reported_and_the_context_stays_usable():
@@ -572,13 +562,63 @@ def test_query_prefill_lse_replaces_the_statistics_pass():
     check_anchor_band(ref_raw, case.k[0], s.anchors.cpu().numpy()[0])
 
 
+def test_query_prefill_attention_emits_the_scores_of_its_own_pass():
+    """relaxkv_query_prefill_attention: one call gives the query's causal attention over [context, query] (output and
+    log-normalisers) AND the context scores with those normalisers - the score of the query's real forward pass.  Two
+    requests with a gap between their cache rows; against the oracle's causal attention and its supplied-normaliser
+    scores, and the anchors picked from the emitted scores against the oracle's top-k band."""
+    H, Hkv, D = 16, 4, 128
+    ctx, qn = (1100, 700), (40, 9)
+    offs = [0, 1300]                                   # rows 1140..1299 belong to nobody
+    rows = 1300 + 700 + 9
+    scale = D ** -0.5
+    g = torch.Generator(device="cpu").manual_seed(21)
+    k_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    v_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    q = torch.randn(sum(qn), H, D, generator=g).to(torch.bfloat16).cuda()
+    shape = B().Shape(H, Hkv, D, list(ctx), list(qn), scale)
+    ext = B().Shape(H, Hkv, D, [c + n for c, n in zip(ctx, qn)], list(qn), scale)
+    ws = torch.empty(B().relaxkv_workspace_bytes(ext, 1) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.zeros_like(q)
+    lse = torch.zeros(H, sum(qn), dtype=torch.float32, device="cuda")
+    raw = torch.zeros(sum(ctx), dtype=torch.float32, device="cuda")
+    B().relaxkv_query_prefill_attention(shape, B().CacheView(k_all, v_all, offs), q, out, lse, raw, ws)
+    assert_status_ok()
+    k_anchor = [B().relaxkv_anchor_count(t, 0.15) for t in ctx]
+    anchors = torch.zeros(1, sum(k_anchor), dtype=torch.int32, device="cuda")
+    B().relaxkv_select_topk(shape, 1, k_anchor, raw.view(1, -1), anchors)
+    assert_status_ok()
+    lo_q = lo_t = lo_k = 0
+    for b in range(2):
+        T, Qn = ctx[b], qn[b]
+        kb = inputs.bf16_bits(k_all[offs[b]:offs[b] + T + Qn].contiguous())
+        vb = inputs.bf16_bits(v_all[offs[b]:offs[b] + T + Qn].contiguous())
+        qb = inputs.bf16_bits(q[lo_q:lo_q + Qn])
+        ref_out, ref_lse = orc.list_attention(kb, vb, qb, None, None, np.arange(T + Qn), np.arange(T, T + Qn), scale)
+        mx, mean = attention_errors(out[lo_q:lo_q + Qn], ref_out)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (b, mx, mean)
+        np.testing.assert_allclose(lse[:, lo_q:lo_q + Qn].cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+        ref_raw = orc.raw_scores(qb, kb[:T], scale, lse=ref_lse.T)
+        got = raw[lo_t:lo_t + T].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref_raw) <= 1e-3 * ref_raw + 1e-6 / T), np.abs(got / ref_raw - 1).max()
+        assert got.sum() < 1.0                               # part of each row's mass sits on the query's own keys
+        check_anchor_band(ref_raw, k_anchor[b], anchors[0, lo_k:lo_k + k_anchor[b]].cpu().numpy())
+        lo_q, lo_t, lo_k = lo_q + Qn, lo_t + T, lo_k + k_anchor[b]
+    # the attention alone (no scores asked for) gives the same output bits
+    out2 = torch.zeros_like(q)
+    B().relaxkv_query_prefill_attention(shape, B().CacheView(k_all, v_all, offs), q, out2, lse, None, ws)
+    assert_status_ok()
+    assert torch.equal(out, out2)
+
+
 @pytest.mark.parametrize("head_major", [False, True])
 @pytest.mark.parametrize("n_splits", [0, 1, 3])
 def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
     """The pass after the repair loop: query rows (and a single decode token) attend to the cache's own causal
     prefix, read through the cache's strides without a gather.  Three requests in one call, token-major and
     head-major caches with a gap between the requests' rows, against the oracle's explicit-list attention with
-    every position as context."""
+    every position as context.  The gaps hold NaN / Inf bit patterns."""
     H, Hkv, D = 16, 4, 128
     lens, n_tgt = (1500, 300, 2200), (37, 1, 64)                 # the middle request is a decode step: one row
     offs = [0, 1600, 2000]                                        # rows 1500..1599 and 1900..1999 belong to nobody
@@ -586,6 +626,12 @@ def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
     g = torch.Generator(device="cpu").manual_seed(5)
     k_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
     v_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    # the rows that belong to nobody hold what an uninitialised slot may hold: NaN and infinities (plain data; the
+    # last tile of every request reaches into them, and a masked key must not let them through)
+    for lo_gap, hi_gap in ((1500, 1600), (1900, 2000), (4200, 4300)):
+        k_all[lo_gap:hi_gap] = float("nan")
+        v_all[lo_gap:hi_gap:2] = float("nan")
+        v_all[lo_gap + 1:hi_gap:2] = float("inf")
     if head_major:
         k_all = k_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
         v_all = v_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
@@ -594,17 +640,13 @@ def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
     tgt = [np.arange(t - n, t, dtype=np.int32) for t, n in zip(lens, n_tgt)]
     tgt_pos = torch.from_numpy(np.concatenate(tgt)).cuda()
     tgt_cu = torch.tensor(np.concatenate([[0], np.cumsum(n_tgt)]).astype(np.int32)).cuda()
-    shape = B().Shape(H, Hkv, D, list(lens), None, D ** -0.5)
+    shape = B().Shape(H, Hkv, D, list(lens), None, D ** -0.5, attention_ctx_splits=n_splits)
     ws = torch.empty(B().relaxkv_workspace_bytes(shape, 1) + 256, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 256:]
     out = torch.zeros_like(q)
     lse = torch.zeros(H, q.shape[0], dtype=torch.float32, device="cuda")
-    B().relaxkv_debug_set_attention_splits(n_splits)
-    try:
-        B().relaxkv_cache_attention(shape, B().CacheView(k_all, v_all, offs), q, tgt_pos, tgt_cu, list(n_tgt), out, ws, lse_out=lse)
-        assert_status_ok()
-    finally:
-        B().relaxkv_debug_set_attention_splits(0)
+    B().relaxkv_cache_attention(shape, B().CacheView(k_all, v_all, offs), q, tgt_pos, tgt_cu, list(n_tgt), out, ws, lse_out=lse)
+    assert_status_ok()
     lo = 0
     for b in range(3):
         kb = inputs.bf16_bits(k_all[offs[b]:offs[b] + lens[b]].contiguous())
@@ -623,10 +665,28 @@ def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
     assert st == B().ERR_BAD_INDEX
 
 
-def test_head_sharded_selection_on_one_gpu():
-    """The head-sharded selection path, its ranks run one after the other on this GPU (their kernels never wait
-    on one another): partial scores of the two KV-head shards average to the unsharded scores, and the anchors
-    computed from the combined scores are those of the unsharded call."""
+def _one_rank_group():
+    """A process group of this one process on the GPU (NCCL): the all-reduce of the sharded path runs for real,
+    over a single rank."""
+    import socket
+    import torch.distributed as dist
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    return dist
+
+
+def test_head_sharded_path_on_one_gpu():
+    """The KV-head-sharded layout, its two ranks run one after the other on this GPU (their kernels never wait on
+    one another).  Selection: each shard's partial scores go through sharded.combine_partial_scores - the all-reduce
+    (over this process alone, so the other shard's partial is added beforehand, which is what the reduction would
+    deliver) and the library's scaling kernel, on a stream of its own - and must average to the unsharded scores;
+    the anchors from the combined scores are those of the unsharded call.  Repair: gather, attention and the cache
+    update on each shard's own heads (cache views k[:, lo:hi], H/N query heads) must equal the oracle's result for
+    those heads, and the two shards' cache updates together the unsharded update, bit for bit."""
     from paper_2609_33503_b200 import sharded
     from paper_2609_33503_b200.pipeline import RepairSession
     case = Case(small_llama(n_layers=2, ctx=(1536,), q=(24,)))
@@ -634,24 +694,134 @@ def test_head_sharded_selection_on_one_gpu():
     full = case.make_session()
     full.score_select(case.q_layers, case.cache_views())
     world = 2
-    parts = []
+    side = torch.cuda.Stream()
+    sessions, parts = [], []
     for rank in range(world):
         kv_lo, kv_hi, q_lo, q_hi = sharded.head_shard(w.n_q_heads, w.n_kv_heads, world, rank)
         s = RepairSession(q_hi - q_lo, kv_hi - kv_lo, w.head_dim, w.ctx_lens, w.q_lens, w.n_layers, case.k,
                           device=case.device, softmax_scale=case.scale)
         qs = [q[:, q_lo:q_hi].contiguous() for q in case.q_layers]
         views = [B().CacheView(k[:, kv_lo:kv_hi], v[:, kv_lo:kv_hi], [0]) for k, v in zip(case.k_cache, case.v_cache)]
-        sharded.sharded_score_select(s, qs, views, world=1)          # world=1: no process group on this machine
+        B().relaxkv_score_select(s.shape, qs, views, s.k, s.raw, None, s.workspace)       # the shard's partial scores
+        sessions.append(s)
         parts.append(s.raw.clone())
-    combined = (parts[0] + parts[1]) / world
+    torch.cuda.synchronize()
+    dist = _one_rank_group()
+    try:
+        for rank in range(world):
+            s = sessions[rank]
+            s.raw.copy_(parts[0] + parts[1])          # what the all-reduce over two ranks delivers to this rank
+            torch.cuda.synchronize()
+            sharded.combine_partial_scores(s, world, stream=side)
+            B().relaxkv_select_topk(s.shape, s.n_layers, s.k, s.raw, s.anchors, stream=side)
+        side.synchronize()
+    finally:
+        dist.destroy_process_group()
     assert_status_ok()
-    torch.testing.assert_close(combined, full.raw, rtol=2e-5, atol=1e-9)
-    s0 = RepairSession(w.n_q_heads // world, w.n_kv_heads // world, w.head_dim, w.ctx_lens, w.q_lens, w.n_layers, case.k,
-                       device=case.device, softmax_scale=case.scale)
-    anchors = torch.empty_like(full.anchors)
-    B().relaxkv_select_topk(s0.shape, w.n_layers, case.k, combined, anchors)
+    for s in sessions:
+        torch.testing.assert_close(s.raw, full.raw, rtol=2e-5, atol=1e-9)
+        assert torch.equal(s.anchors, sessions[0].anchors)            # every rank selects the same anchors
+        for l in range(w.n_layers):
+            check_anchor_band(case.raw[(l, 0)], case.k[0], s.anchors[l].cpu().numpy())
+    # ---- the repair half on each shard's heads, on the oracle's sets ----
+    k_upd = [k.clone() for k in case.k_cache]
+    v_upd = [v.clone() for v in case.v_cache]
+    for rank in range(world):
+        kv_lo, kv_hi, q_lo, q_hi = sharded.head_shard(w.n_q_heads, w.n_kv_heads, world, rank)
+        s = sessions[rank]
+        s.build_active_sets(case.anchors_tensor())
+        n_u, n_r = s.counts()
+        for l in range(w.n_layers):
+            f = case.fresh[l]
+            qn, kn, vn = f.q_new[:, q_lo:q_hi].contiguous(), f.k_new[:, kv_lo:kv_hi].contiguous(), f.v_new[:, kv_lo:kv_hi].contiguous()
+            view = B().CacheView(case.k_cache[l][:, kv_lo:kv_hi], case.v_cache[l][:, kv_lo:kv_hi], [0])
+            rows = sum(n_u) + 128
+            kc = torch.empty(rows, kv_hi - kv_lo, w.head_dim, dtype=torch.bfloat16, device=case.device)
+            vc = torch.empty_like(kc)
+            s.gather(l, view, kn, vn, n_u, kc, vc)
+            kt, vt = orc.mix_context(case.req_k(l, 0)[:, kv_lo:kv_hi].copy(), case.req_v(l, 0)[:, kv_lo:kv_hi].copy(),
+                                     inputs.bf16_bits(kn), inputs.bf16_bits(vn), case.sets[0].u_pos, case.sets[0].ranks(l))
+            np.testing.assert_array_equal(inputs.bf16_bits(kc[:n_u[0]]), kt)
+            np.testing.assert_array_equal(inputs.bf16_bits(vc[:n_u[0]]), vt)
+            out = torch.zeros_like(qn)
+            s.attention(l, view, qn, kn, vn, out, n_r[l], n_u)
+            assert_status_ok()
+            ref, _ = orc.repair_attention(case.req_k(l, 0)[:, kv_lo:kv_hi].copy(), case.req_v(l, 0)[:, kv_lo:kv_hi].copy(),
+                                          inputs.bf16_bits(qn), inputs.bf16_bits(kn), inputs.bf16_bits(vn),
+                                          case.sets[0].u_pos, case.sets[0].ranks(l), case.scale)
+            mx, mean = attention_errors(out, ref)
+            assert mx <= MAX_ABS and mean <= MEAN_ABS, (rank, l, mx, mean)
+            s.scatter(l, B().CacheView(k_upd[l][:, kv_lo:kv_hi], v_upd[l][:, kv_lo:kv_hi], [0]), kn, vn, n_r[l])
+    assert_status_ok()
+    whole = case.make_session()
+    whole.build_active_sets(case.anchors_tensor())
+    _, n_r = whole.counts()
     for l in range(w.n_layers):
-        check_anchor_band(case.raw[(l, 0)], case.k[0], anchors[l].cpu().numpy())
+        k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+        whole.scatter(l, B().CacheView(k2, v2, [0]), case.fresh[l].k_new, case.fresh[l].v_new, n_r[l])
+        assert torch.equal(k2, k_upd[l]) and torch.equal(v2, v_upd[l])
+
+
+def test_one_chunk_reading_fresh_states_equal_to_the_cache():
+    """With a single chunk nothing precedes the chunk, so recomputing a token gives back its cached K/V.  Then
+    (i) the cache update leaves the cache bit-identical, (ii) attention over the mixed fresh/cached context equals
+    attention over the cache alone bit for bit, and (iii) at an anchor ratio of 100 % the output is dense causal
+    attention over the cache, i.e. a plain prefix prefill (checked against causal attention in float64)."""
+    for ratio in (0.3, 1.0):
+        w = small_qwen(n_layers=2, ctx=(900,), q=(16,)).replace(ratio=ratio)
+        case = Case(w)
+        s = case.make_session()
+        s.build_active_sets(case.anchors_tensor())
+        n_u, n_r = s.counts()
+        for l in range(w.n_layers):
+            pos = torch.from_numpy(case.sets[0].positions(l).astype(np.int64)).to(case.device)
+            f = case.fresh[l]
+            k_same, v_same = case.k_cache[l][pos].contiguous(), case.v_cache[l][pos].contiguous()
+            view = case.cache_views()[l]
+            mixed = torch.zeros_like(f.q_new)
+            s.attention(l, view, f.q_new, k_same, v_same, mixed, n_r[l], n_u)
+            alone = torch.zeros_like(f.q_new)
+            s.attention(l, view, f.q_new, None, None, alone, n_r[l], n_u)
+            assert_status_ok()
+            assert torch.equal(mixed, alone)
+            k2, v2 = case.k_cache[l].clone(), case.v_cache[l].clone()
+            s.scatter(l, B().CacheView(k2, v2, [0]), k_same, v_same, n_r[l])
+            assert torch.equal(k2, case.k_cache[l]) and torch.equal(v2, case.v_cache[l])
+            if ratio == 1.0:
+                assert n_r[l] == [900] and n_u == [900]
+                G = w.group
+                q64 = f.q_new.double().cpu().permute(1, 0, 2).unsqueeze(0)
+                k64 = case.k_cache[l].double().cpu().repeat_interleave(G, dim=1).permute(1, 0, 2).unsqueeze(0)
+                v64 = case.v_cache[l].double().cpu().repeat_interleave(G, dim=1).permute(1, 0, 2).unsqueeze(0)
+                ref = torch.nn.functional.scaled_dot_product_attention(q64, k64, v64, is_causal=True, scale=case.scale)[0].permute(1, 0, 2)
+                d = (mixed.double().cpu() - ref).abs()
+                assert d.max().item() <= MAX_ABS and d.mean().item() <= MEAN_ABS
+
+
+def test_list_call_with_more_context_than_its_host_bound_is_reported():
+    """Explicit lists whose true context count exceeds the host bound: the rows past the bound have no entry in the
+    fresh-row map, so the gather must not use one (it zero-fills them) and the status word reports the overflow."""
+    case = Case(small_llama(n_layers=1, ctx=(512,), q=(8,)))
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    sets = case.sets[0]
+    ctx_list, tgt_list = sets.u_pos.astype(np.int32), sets.positions(0).astype(np.int32)
+    f = case.fresh[0]
+    ctx_pos, ctx_cu, _ = _pack([ctx_list], case.device)
+    tgt_pos, tgt_cu, _ = _pack([tgt_list], case.device)
+    s.workspace.view(torch.int32).fill_(0x7fffff00)            # stale words a trusting kernel would index with
+    out = torch.zeros_like(f.q_new)
+    B().relaxkv_list_attention(s.shape, case.cache_views()[0], f.q_new, f.k_new, f.v_new, ctx_pos, ctx_cu, tgt_pos, tgt_cu,
+                               [len(tgt_list)], [len(ctx_list) - 40], out, s.workspace)
+    st, detail = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX, (st, detail)
+    out2 = torch.zeros_like(f.q_new)                           # the context stays usable: the same call with a true bound
+    B().relaxkv_list_attention(s.shape, case.cache_views()[0], f.q_new, f.k_new, f.v_new, ctx_pos, ctx_cu, tgt_pos, tgt_cu,
+                               [len(tgt_list)], [len(ctx_list)], out2, s.workspace)
+    assert_status_ok()
+    ref, _ = case.oracle_attention(0, 0)
+    mx, mean = attention_errors(out2, ref)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS
 
 
 # ------------------------------------------------ other head geometries and cache layouts ----

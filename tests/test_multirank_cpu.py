@@ -55,7 +55,14 @@ def _shard_worker(rank, world, port, out):
     # the rank's partial score: the oracle on its own heads only (stands in for the CUDA kernels on a CPU machine)
     local = orc.raw_scores(inputs.bf16_bits(q[:, q_lo:q_hi]), inputs.bf16_bits(k[:, kv_lo:kv_hi]), scale)
     t = torch.from_numpy(local).clone().view(1, -1)
-    sharded.combine_partial_scores(t, world)
+
+    class HostSession:            # the fields combine_partial_scores reads
+        raw, n_layers, shape = t, 1, None
+
+    def scale_on_host(session, factor):   # stands in for relaxkv_scale_scores, like the oracle does for the scoring
+        session.raw.mul_(factor)
+
+    sharded.combine_partial_scores(HostSession, world, scale_fn=scale_on_host)
     full = orc.raw_scores(inputs.bf16_bits(q), inputs.bf16_bits(k), scale)
     out[rank] = (float(np.abs(t.numpy()[0] - full).max() / full.max()), orc.topk(t.numpy()[0], 58).tolist() == orc.topk(full, 58).tolist())
     dist.barrier()
@@ -74,3 +81,21 @@ def test_head_sharded_scores_combine_to_the_full_score():
     for r in range(world):
         err, same = out[r]
         assert err < 1e-12 and same
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_several_gpus():
+    """`bench.py --gpus N` without a launcher around it starts N local ranks itself (torch.distributed.run,
+    rendezvous on 127.0.0.1).  Driven here with a stand-in job and gloo: the printed line must come from rank 0,
+    count two ranks, carry the slowest rank's time and the whole-job value."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-ranks"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["ms_per_step"] == 15.0 and d["backend"] == "gloo"
+    assert abs(d["value"] - 2 * 2.0e12 / 15e-3 / 1e12) < 1e-9
