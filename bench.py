@@ -226,27 +226,58 @@ class GpuJob:
         # gather + attention + scatter
         self.launches_per_step = 4 * ((L + 47) // 48) + 1 + 5 + 3 * L
 
+    kv_reps = 10          # timed replays of the gather / scatter graphs (--kv-reps)
+
+    def _time_graph(self, enqueue, reps: int = 0):
+        """ms per replay of a CUDA graph that holds the kernels `enqueue` launches: the kernels run back to back with
+        no host work between them, so the figure is the kernels' own duration (a CUDA-event pair around one
+        25-microsecond call also holds the host's launch work whenever the GPU has run dry)."""
+        side = torch.cuda.Stream(device=self.device)
+        side.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(side):
+            enqueue()                                   # first calls outside the capture (one-time lookups)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                enqueue()
+        torch.cuda.current_stream(self.device).wait_stream(side)
+        torch.cuda.synchronize()
+        reps = reps or self.kv_reps
+        for _ in range(min(3, reps)):
+            g.replay()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b_.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b_) / reps
+
     def time_gather(self, mode):
-        """One pass over the layers of relaxkv_gather_kv alone (same kernel and arguments as inside the
-        attention call), CUDA events around each call; other layers' traffic keeps L2 cold."""
+        """One pass over the layers of relaxkv_gather_kv alone (same kernel and arguments as inside the attention
+        call), all launches in one CUDA graph; the layers' inputs together exceed L2."""
         w, s = self.w, self.s
         n_u, n_r = s.counts()
         rows = (sum(n_u) if mode == self.B.CTX_UNION else int(self.ctx_cu[-1])) + 128
         kc = torch.empty(rows, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device=self.device)
         vc = torch.empty_like(kc)
-        total = 0.0
-        for rep in range(2):
-            evs = []
+
+        def enqueue():
             for l in range(w.n_layers):
                 f = self.fresh[l]
-                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
                 s.gather(l, self.views[l], f[1], f[2], n_u, kc, vc, mode=mode)
-                b_.record()
-                evs.append((a, b_))
-            torch.cuda.synchronize()
-            total = sum(a.elapsed_time(b_) for a, b_ in evs)
-        return total
+        return self._time_graph(enqueue)
+
+    def time_scatter(self):
+        """One pass over the layers of relaxkv_scatter_kv alone, all launches in one CUDA graph (the update is
+        idempotent, so replaying it changes nothing)."""
+        s = self.s
+        n_u, n_r = s.counts()
+
+        def enqueue():
+            for l in range(self.w.n_layers):
+                f = self.fresh[l]
+                s.scatter(l, self.views[l], f[1], f[2], n_r[l])
+        return self._time_graph(enqueue)
 
     def time_attention_stream(self, mode, reps: int):
         """ms per pass over the layers' attention calls when `reps` passes are queued back to back with no host
@@ -313,6 +344,7 @@ def measure(job: GpuJob, full_prefix: bool, steps: int, warmup: int, peaks, devi
     phase_ms = {k: v / steps for k, v in phase_ms.items()}
     ms_per_step = elapsed_ms / steps
     gather_ms = job.time_gather(mode)
+    scatter_ms = job.time_scatter()
     L = w.n_layers
     flops = job.flops(full_prefix)
     kv_row = w.n_kv_heads * w.head_dim * 2
@@ -344,8 +376,13 @@ def measure(job: GpuJob, full_prefix: bool, steps: int, warmup: int, peaks, devi
                  "edges": int(sum(job.edges)), "edges_full_prefix": int(sum(job.edges_full))},
         "attention_tflops": round(attn_tflops, 2),
         "attention_frac_of_sustained_peak": round(attn_tflops / peaks["bf16_tflops_sustained"], 4),
-        "scatter_gbs": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9, 1),
-        "scatter_frac_hbm": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "scatter_us": round(scatter_ms * 1e3, 1),
+        "scatter_gbs": round(scatter_bytes / (scatter_ms * 1e-3) / 1e9, 1),
+        "scatter_frac_hbm": round(scatter_bytes / (scatter_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "scatter_frac_hbm_in_step": round(scatter_bytes / (phase_ms["scatter"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "kv_move_timing": "gather and scatter: all layers' launches replayed from one CUDA graph (kernel durations back to "
+                          "back, inputs larger than L2); *_in_step: CUDA-event pairs around each call inside the step, "
+                          "which also hold the launch gap of a 25-microsecond kernel",
         "gather_us": round(gather_ms * 1e3, 1),
         "gather_gbs": round(gather_bytes / (gather_ms * 1e-3) / 1e9, 1),
         "gather_frac_hbm": round(gather_bytes / (gather_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
@@ -474,7 +511,8 @@ def run_gpu(args):
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "layer_stack_us": round(ms_per_step * 1e3, 1),
         "phases_us": m["phases_us"], "sets": m["sets"],
-        "scatter_gbs": m["scatter_gbs"], "scatter_frac_hbm": m["scatter_frac_hbm"],
+        "scatter_us": m["scatter_us"], "scatter_gbs": m["scatter_gbs"], "scatter_frac_hbm": m["scatter_frac_hbm"],
+        "scatter_frac_hbm_in_step": m["scatter_frac_hbm_in_step"], "kv_move_timing": m["kv_move_timing"],
         "gather_us": m["gather_us"], "gather_gbs": m["gather_gbs"], "gather_frac_hbm": m["gather_frac_hbm"],
         "scoring": m["scoring"],
         "roofline": {"bound": "tensor", "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"],
@@ -839,6 +877,139 @@ def run_dense(args):
     print(json.dumps(out))
 
 
+def run_ttft(args):
+    """The paper's time-to-first-token region on one request with synthetic block weights: the query's forward pass
+    over the naive cache (which emits the context scores of every layer from its own attention - no separate scoring
+    pass), top-k and the repair schedule, the repair loop with the active rows' block work, the query's prefill over
+    the repaired cache, the final norm and output head of the last query row; one further decode step is reported
+    beside it.  Every phase runs in the library's kernels; the sequencing is query_pass.QueryPass and
+    layer_loop.LayerLoop."""
+    from paper_2609_33503_b200 import binding as B
+    from paper_2609_33503_b200.layer_loop import LayerLoop
+    from paper_2609_33503_b200.pipeline import RepairSession
+    from paper_2609_33503_b200.query_pass import QueryPass
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    w = make_workload(args)
+    if w.n_req != 1:
+        raise SystemExit("--ttft times one request")
+    blk = inputs.LLAMA31_8B_BLOCK if w.n_q_heads == 32 else inputs.QWEN3_14B_BLOCK
+    vocab = 128256 if w.n_q_heads == 32 else 151936
+    if args.workload == "tiny":
+        blk, vocab = inputs.BlockShape(hidden=256, inter=512), 4096
+    L, T, Q = w.n_layers, w.ctx_lens[0], w.q_lens[0]
+    rows = T + Q + 2
+    k = [B.relaxkv_anchor_count(T, w.ratio)]
+    naive, repaired, weights = [], [], []
+    for l in range(L):
+        _, kk, vv = inputs.layer_qkv(w, l, 0, device)
+        bufs = []
+        for _ in range(2):
+            ka = torch.zeros(rows, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device=device)
+            va = torch.zeros_like(ka)
+            ka[:T], va[:T] = kk, vv
+            bufs.append(B.CacheView(ka, va, [0]))
+        naive.append(bufs[0]); repaired.append(bufs[1])
+        weights.append(inputs.block_weights(w, blk, l, device))
+    g = torch.Generator(device=device).manual_seed(77)
+    hq0 = torch.randn(Q, blk.hidden, device=device, generator=g).to(torch.bfloat16)       # the query tokens' input rows
+    h_tok = torch.randn(1, blk.hidden, device=device, generator=g).to(torch.bfloat16)     # the first decoded token's
+    w_final = (1.0 + 0.1 * torch.randn(blk.hidden, device=device, generator=g)).to(torch.bfloat16)
+    w_head = (torch.randn(vocab, blk.hidden, device=device, generator=g) * blk.hidden ** -0.5).to(torch.bfloat16)
+    logits = torch.empty(1, vocab, dtype=torch.bfloat16, device=device)
+    s = RepairSession(w.n_q_heads, w.n_kv_heads, w.head_dim, [T], [Q], L, k, device=device)
+    qp = QueryPass(w.n_q_heads, w.n_kv_heads, w.head_dim, [T], [Q], blk, device=device)
+    # untimed pass to learn U (the rows whose input representations the repair loop starts from)
+    qp.prefill(hq0, weights, naive, scores_out=s.raw)
+    B.relaxkv_select_topk(s.shape, L, s.k, s.raw, s.anchors)
+    s.build_active_sets()
+    n_u, n_r = s.counts()
+    u_pos = s.u_pos.cpu().numpy()[:n_u[0]].astype(np.int64)
+    h0 = inputs.input_representations(w, blk, 0, torch.from_numpy(u_pos), device).contiguous()
+    loop = LayerLoop(s, blk, n_u[0])
+    r_rank, r_cu = s.r_rank.cpu().numpy(), s.r_cu.cpu().numpy()
+    edges = sum(int(r_rank[r_cu[i]:r_cu[i + 1]].astype(np.int64).sum() + (r_cu[i + 1] - r_cu[i])) for i in range(L))
+
+    # The query passes and the decode step are some 600 short launches each: replayed from CUDA graphs, so that the
+    # host's launch work (tens of microseconds per call from Python) does not set their time.
+    qp.decode_positions(0)
+
+    def graph_of(fn):
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(torch.cuda.current_stream(device))
+        with torch.cuda.stream(side):
+            fn()
+            g_ = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_, stream=side):
+                fn()
+        torch.cuda.current_stream(device).wait_stream(side)
+        torch.cuda.synchronize()
+        return g_
+
+    if args.no_graphs:
+        class Eager:
+            def __init__(self, fn): self.fn = fn
+            def replay(self): self.fn()
+        graph_of = Eager
+    g_scores = graph_of(lambda: qp.prefill(hq0, weights, naive, scores_out=s.raw))
+    g_prefill = graph_of(lambda: qp.output_head(qp.prefill(hq0, weights, repaired), w_final, w_head, logits))
+    g_decode = graph_of(lambda: qp.output_head(qp.decode(h_tok, weights, repaired), w_final, w_head, logits))
+
+    def step(ev=None):
+        def rec(name, fn):
+            if ev is None:
+                fn(); return
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b_.record(); ev.append((name, a, b_))
+        rec("query_pass_with_scores", g_scores.replay)
+        rec("select_and_schedule", lambda: (B.relaxkv_select_topk(s.shape, L, s.k, s.raw, s.anchors), s.build_active_sets()))
+        s.counts()
+        rec("repair_loop", lambda: loop.run(h0, weights, repaired))
+        rec("query_prefill_and_first_token_head", g_prefill.replay)
+        rec("decode_step", g_decode.replay)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    check_status(B)
+    sampler = ClockSampler(0).start()
+    time.sleep(0.3)
+    ev = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step(ev)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    check_status(B)
+    phase = {}
+    for name, a, b_ in ev:
+        phase[name] = phase.get(name, 0.0) + a.elapsed_time(b_) / args.steps
+    total = t0.elapsed_time(t1) / args.steps
+    ttft = total - phase["decode_step"]
+    weight_bytes = sum(v.numel() * 2 for wl in weights for k_, v in wl.items() if k_ != "w_gate_up") + w_head.numel() * 2
+    peaks = load_peaks()
+    out = {"metric": "ttft_ms", "value": round(ttft, 3), "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": round(total, 3), "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic",
+           "config": {"workload": w.name, "n_layers": L, "ctx_len": T, "query_len": Q, "anchor_ratio": w.ratio,
+                      "block": dataclass_dict(blk), "vocab": vocab, "l2": "inputs larger than L2"},
+           "phases_us": {k_: round(v * 1e3, 1) for k_, v in phase.items()},
+           "region": "query pass over the naive cache with fused scoring + selection + repair loop (block work, repair "
+                     "attention, cache update) + query prefill over the repaired cache + final norm and output head; "
+                     "decode_step (one more token through all layers + head) is reported beside it, not inside value",
+           "launch": "eager calls" if args.no_graphs else "query passes and decode step replayed from CUDA graphs; the repair loop, "
+                     "whose launch sizes depend on the selected sets, is launched call by call",
+           "sets": {"ctx_ratio": round(n_u[0] / T, 4), "active_ratio": round(sum(x[0] for x in n_r) / (L * T), 4), "edges": int(edges)},
+           "decode_step": {"us": round(phase["decode_step"] * 1e3, 1), "weight_bytes": int(weight_bytes),
+                           "weights_gbs": round(weight_bytes / (phase["decode_step"] * 1e-3) / 1e9, 1),
+                           "frac_hbm": round(weight_bytes / (phase["decode_step"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                           "note": "bytes = every block weight and the output head once; K/V reads (2 x 40 x 67 MB) not counted"},
+           "clocks": clocks}
+    print(json.dumps(out))
+
+
 def dataclass_dict(x):
     import dataclasses
     return dataclasses.asdict(x)
@@ -979,12 +1150,18 @@ def main():
                          "rotary embedding, MLP with synthetic weights); prints its own JSON line")
     ap.add_argument("--query-attention", action="store_true",
                     help="time the user query's prefill rows and a decode step over the context cache (same kernel, context split)")
+    ap.add_argument("--ttft", action="store_true",
+                    help="time the whole time-to-first-token region with synthetic block weights: query pass with fused "
+                         "scoring, selection, repair loop, query prefill, output head (+ one decode step)")
+    ap.add_argument("--no-graphs", action="store_true", help="--ttft: launch the query passes and the decode step call by call")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the other benchmark configurations after the headline workload")
     ap.add_argument("--cpu-rows", type=int, default=256)
+    ap.add_argument("--kv-reps", type=int, default=10, help="timed replays of the gather-only and scatter-only CUDA graphs")
     ap.add_argument("--selftest-ranks", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    GpuJob.kv_reps = max(1, args.kv_reps)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # no launcher around us: start the ranks ourselves, one process per GPU
         raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
@@ -996,6 +1173,8 @@ def main():
         run_query_attention(args)
     elif args.dense:
         run_dense(args)
+    elif args.ttft:
+        run_ttft(args)
     elif args.config != "relaxkv":
         run_list_config(args)
     else:

@@ -30,6 +30,13 @@
  *             the device can see (an index out of range, a count above its host bound, a bounded
  *             wait that expired) are recorded in a device status word - the kernel skips the
  *             offending work and returns normally - and are read with relaxkv_read_device_status.
+ *             The first problem recorded stays until it is read.  After an expired wait (RELAXKV_ERR_TIMEOUT)
+ *             the tensor-core kernels of later calls on that device return at once without writing their
+ *             outputs, until the status word has been read (and thereby cleared): a caller that sees garbage
+ *             should read the status word first.
+ * Threads.    Calls may be made from several host threads; the per-device values the library looks up once
+ *             (device addresses, attribute opt-ins) are published with atomics.  The status word is per device,
+ *             not per thread or stream.
  * Precision.  bf16 inputs, fp32 accumulation and softmax, probabilities rounded to bf16 before the
  *             P*V product, bf16 outputs.
  */

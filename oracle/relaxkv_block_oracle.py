@@ -53,3 +53,36 @@ def compact_rows(h: np.ndarray, ranks_l: np.ndarray, ranks_next: np.ndarray) -> 
     keep = np.isin(ranks_l, ranks_next)
     assert keep.sum() == len(ranks_next)
     return h[keep]
+
+
+def decoder_block(h: np.ndarray, W: dict, n_q_heads: int, n_kv_heads: int, head_dim: int, positions: np.ndarray,
+                  eps: float, theta: float, attend, store=lambda t: t) -> np.ndarray:
+    """One pre-norm decoder block on the given rows, written out operation by operation in the order the paper's
+    loop runs them (Algorithm 1, steps 14-22 for the active targets; the same block serves the query's prefill rows
+    and a decode token): input RMSNorm, Q/K/V projections, per-head Q/K RMSNorm when the weights have one, rotary
+    embedding at `positions`, attention, output projection + residual, post-attention RMSNorm, SwiGLU MLP + residual.
+
+    h [rows, hidden] float64; W: float64 weights (w_in_norm, wq, wk, wv, optional w_q_norm / w_k_norm, wo, w_post_norm,
+    w_gate_up = [gate; up] stacked, w_down).  attend(q [rows, H, D], k [rows, Hkv, D], v [rows, Hkv, D]) -> o [rows, H, D]
+    is the attention of these rows (the caller decides what they see).  `store` is applied wherever a tensor is
+    written to memory between two operations (identity: pure float64; a bf16 rounding models bf16 storage)."""
+    n = h.shape[0]
+    H, Hkv, D = n_q_heads, n_kv_heads, head_dim
+    x = store(rmsnorm(h, W["w_in_norm"], eps))
+    q = store(linear(x, W["wq"])).reshape(n, H, D)
+    k = store(linear(x, W["wk"])).reshape(n, Hkv, D)
+    v = store(linear(x, W["wv"])).reshape(n, Hkv, D)
+    if "w_q_norm" in W:
+        q = store(rmsnorm(q.reshape(n * H, D), W["w_q_norm"], eps)).reshape(n, H, D)
+        k = store(rmsnorm(k.reshape(n * Hkv, D), W["w_k_norm"], eps)).reshape(n, Hkv, D)
+    q, k = store(rope(q, positions, theta)), store(rope(k, positions, theta))
+    o = store(attend(q, k, v)).reshape(n, H * D)
+    a = store(linear(o, W["wo"], h))
+    x2 = store(rmsnorm(a, W["w_post_norm"], eps))
+    m = store(swiglu(linear(x2, W["w_gate_up"])))
+    return store(linear(m, W["w_down"], a))
+
+
+def output_head(h_row: np.ndarray, w_final_norm: np.ndarray, w_head: np.ndarray, eps: float, store=lambda t: t) -> np.ndarray:
+    """Logits of one row per request: final RMSNorm, then the output projection [vocab, hidden]."""
+    return store(linear(store(rmsnorm(h_row, w_final_norm, eps)), w_head))

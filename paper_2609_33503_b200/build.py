@@ -17,6 +17,12 @@ LIB = os.path.join(HERE, "librelaxkv.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
+# RELAXKV_NVTX=1: compile NVTX ranges into every C-ABI call and kernel launch (the header-only NVTX v3 of the toolkit);
+# objects of the two flavours are kept apart
+NVTX = os.environ.get("RELAXKV_NVTX", "0") not in ("", "0")
+if NVTX:
+    FLAGS += ["-DRELAXKV_NVTX"]
+    OBJ = os.path.join(HERE, "build_nvtx")
 
 
 def sources():
@@ -53,7 +59,7 @@ def build(force: bool = False, verbose: bool = False, ptxas_v: bool = False) -> 
     objs = [os.path.join(OBJ, s[:-3] + ".o") for s in sources()]
     if jobs or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
         tmp = LIB + f".tmp{os.getpid()}"
-        subprocess.check_call([NVCC, "-shared", "-o", tmp, *objs])
+        subprocess.check_call([NVCC, "-shared", "-o", tmp, *objs, *(["-ldl"] if NVTX else [])])
         os.replace(tmp, LIB)
     return LIB
 

@@ -71,6 +71,7 @@ extern "C" size_t relaxkv_workspace_bytes(const relaxkv_shape* shape, int32_t n_
 
 extern "C" relaxkv_status relaxkv_read_device_status(int32_t* h_status_out, int32_t* h_detail_out,
                                                      relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_read_device_status");
   if (!h_status_out) return RELAXKV_ERR_INVALID_ARG;
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;

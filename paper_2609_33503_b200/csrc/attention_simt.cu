@@ -100,6 +100,7 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention_simt(
     const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
     int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
     void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_sparse_ctx_attention_simt");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   AttnPlan plan;
   relaxkv_status rc = prepare_attention(shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer,

@@ -669,6 +669,7 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention(
     const int32_t* u_pos, const int32_t* u_cu, const int32_t* r_rank, const int32_t* r_cu_layer,
     int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
     void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_sparse_ctx_attention");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   AttnPlan plan;
   relaxkv_status rc = prepare_attention(shape, mode, cache, q_new, k_new, v_new, u_pos, u_cu, r_rank, r_cu_layer,
@@ -681,6 +682,7 @@ extern "C" relaxkv_status relaxkv_sparse_ctx_attention(
 }
 
 extern "C" relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_debug_wait_timeout");
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
   wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(st);
@@ -693,6 +695,7 @@ extern "C" relaxkv_status relaxkv_list_attention(
     const int32_t* ctx_pos, const int32_t* ctx_cu, const int32_t* tgt_pos, const int32_t* tgt_cu,
     int64_t n_target_rows, const int32_t* h_max_targets, const int32_t* h_max_ctx,
     void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_list_attention");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
@@ -744,6 +747,7 @@ extern "C" relaxkv_status relaxkv_cache_attention(
     const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q_new,
     const int32_t* tgt_pos, const int32_t* tgt_cu, int64_t n_target_rows, const int32_t* h_max_targets,
     void* out, float* lse_out, void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_cache_attention");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;

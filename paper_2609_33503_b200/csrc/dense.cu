@@ -178,6 +178,7 @@ using namespace relaxkv;
 
 extern "C" relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64_t n_rows, int32_t n_cols,
                                           float eps, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_rmsnorm");
   if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || !(eps >= 0.f)) return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_cols < 8 || (n_cols % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
@@ -196,6 +197,7 @@ extern "C" relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, voi
 
 extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
                                        float theta, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_rope");
   if (!x || !positions || !aligned16(x) || !(theta > 1.f)) return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_heads < 1 || (head_dim != 64 && head_dim != 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
@@ -206,6 +208,7 @@ extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads,
 }
 
 extern "C" relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t n_rows, int32_t n_inter, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_swiglu");
   if (!gate_up || !out || !aligned16(gate_up) || !aligned16(out)) return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_inter < 8 || (n_inter % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   if (n_rows == 0) return RELAXKV_OK;
@@ -218,6 +221,7 @@ extern "C" relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t
 extern "C" relaxkv_status relaxkv_target_positions(const relaxkv_shape* shape, const int32_t* u_pos, const int32_t* u_cu,
                                                    const int32_t* r_rank, const int32_t* r_cu_layer,
                                                    const int32_t* h_max_targets, int32_t* positions_out, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_target_positions");
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if (!u_pos || !u_cu || !r_rank || !r_cu_layer || !h_max_targets || !positions_out) return RELAXKV_ERR_INVALID_ARG;
@@ -241,6 +245,7 @@ extern "C" relaxkv_status relaxkv_target_positions(const relaxkv_shape* shape, c
 extern "C" relaxkv_status relaxkv_carry_rows(const relaxkv_shape* shape, const void* h_in, void* h_out, int32_t n_cols,
                                              const int32_t* r_rank, const int32_t* r_cu_layer, const int32_t* r_cu_next,
                                              const int32_t* h_max_next, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_carry_rows");
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if (!h_in || !h_out || !r_rank || !r_cu_layer || !r_cu_next || !h_max_next || !aligned16(h_in) || !aligned16(h_out))

@@ -467,11 +467,13 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
 
 extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
                                          int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_linear");
   return launch_gemm(x, weight, residual, y, n_rows, n_out, n_in, 0, stream_);
 }
 
 extern "C" relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weight_tiled, void* y, int64_t n_rows,
                                                 int32_t n_inter, int32_t n_in, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_linear_swiglu");
   if (n_inter < 128 || (n_inter % 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   return launch_gemm(x, weight_tiled, nullptr, y, n_rows, 2 * n_inter, n_in, 1, stream_);
 }

@@ -1,8 +1,9 @@
 // Projections of a handful of rows (a decode token, the last query row going through the output head): y = x W^T with
 // at most kGemvMaxRows rows of x.  The work is reading W once (HBM-bound: every weight byte meets one to four
-// multiply-adds), so this is a plain streaming kernel, not the 128-row tensor-core GEMM: each warp owns four output
-// features, its lanes stride over K in 16-byte pieces with eight independent weight loads in flight per lane, x stays
-// in L1, and a shuffle tree sums the lanes' partial dot products in a fixed order.  (Algorithm 1 runs "the unchanged
+// multiply-adds), so this is a plain streaming kernel, not the 128-row tensor-core GEMM: each warp owns two output
+// features (16 per block: a 5120-wide projection is 320 blocks, all resident at once), its lanes stride over K in
+// 16-byte pieces with eight independent weight loads in flight per lane, x stays in L1, and a shuffle tree sums the
+// lanes' partial dot products in a fixed order.  (Algorithm 1 runs "the unchanged
 // Transformer block"; after the repair loop the same block serves the decode step of the TTFT region.)
 #include "common.cuh"
 #include "gemv.cuh"
@@ -10,7 +11,7 @@
 namespace relaxkv {
 
 constexpr int kGemvThreads = 256;
-constexpr int kGemvFeatPerWarp = 4;
+constexpr int kGemvFeatPerWarp = 2;        // few features per warp: many blocks, so that enough bytes are in flight
 constexpr int kGemvFeatPerBlock = (kGemvThreads / 32) * kGemvFeatPerWarp;
 
 __device__ __forceinline__ void unpack8_gemv(const uint4& v, float* f) {
@@ -41,7 +42,7 @@ gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, cons
   for (int r = 0; r < R; ++r)
 #pragma unroll
     for (int m = 0; m < M; ++m) acc[r][m] = 0.f;
-#pragma unroll 2
+#pragma unroll 4
   for (int k = lane * 8; k < K; k += 32 * 8) {
     uint4 wv[R];
 #pragma unroll

@@ -104,6 +104,7 @@ extern "C" relaxkv_status relaxkv_score_select(
     const float* const* row_lse_layers, const int32_t* h_k,
     float* raw_scores_out, float* norm_scores_out, int32_t* anchors_out,
     void* workspace, size_t workspace_bytes, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_score_select");
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if (n_layers < 1 || !q_layers || !cache_layers || !h_k || !raw_scores_out || !workspace || !shape->h_q_len)

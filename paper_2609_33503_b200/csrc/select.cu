@@ -157,6 +157,7 @@ using namespace relaxkv;
 extern "C" relaxkv_status relaxkv_select_topk(const relaxkv_shape* shape, int32_t n_layers, const int32_t* h_k,
                                               const float* raw_scores, float* norm_scores_out, int32_t* anchors_out,
                                               relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_select_topk");
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if (n_layers < 1 || !h_k || !raw_scores || !anchors_out) return RELAXKV_ERR_INVALID_ARG;
@@ -169,6 +170,7 @@ extern "C" relaxkv_status relaxkv_select_topk(const relaxkv_shape* shape, int32_
 
 extern "C" relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers, const float* scores,
                                               float* mean_out, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_mean_scores");
   relaxkv_status rc = check_shape(shape);
   if (rc != RELAXKV_OK) return rc;
   if (n_layers < 1 || !scores || !mean_out) return RELAXKV_ERR_INVALID_ARG;

@@ -62,6 +62,15 @@ class QueryPass:
         self.dq, self.dk, self.dv, self.do = e(nb, H, D), e(nb, Hkv, D), e(nb, Hkv, D), e(nb, H, D)
         self.dgu, self.dm = e(nb, 2 * I), e(nb, I)
         self.d_cu = torch.arange(nb + 1, **i32)
+        self._dec_pos = {}
+
+    def decode_positions(self, step: int) -> torch.Tensor:
+        """Device tensor of the decoded token's position per request (T_c + Q_b + step), built once per step index so
+        that `decode` itself performs no host-to-device copy (it can then be captured into a CUDA graph)."""
+        if step not in self._dec_pos:
+            self._dec_pos[step] = torch.tensor([c + q + step for c, q in zip(self.ctx_lens, self.q_lens)],
+                                               dtype=torch.int32, device=self.device)
+        return self._dec_pos[step]
 
     def _block(self, l, w, cache, h, x, a, q, k, v, o, gu, m, h_out, pos, cu, counts, shape, attend, rec):
         blk, D, n = self.blk, self.D, h.shape[0]
@@ -121,7 +130,7 @@ class QueryPass:
         T_c + Q_b + step.  Appends its K/V to the caches and returns the hidden row after the last layer."""
         rec = self._rec(events)
         nb = len(self.ctx_lens)
-        pos = torch.tensor([c + q + step for c, q in zip(self.ctx_lens, self.q_lens)], dtype=torch.int32, device=self.device)
+        pos = self.decode_positions(step)
         h = h_tok
         for l, w in enumerate(weights):
             h_out = self.dh[l % 2]
