@@ -157,7 +157,7 @@ relaxkv_status relaxkv_select_topk(
 
 /*
  * Repair schedule from the per-layer anchors (Section 3.2, definitions of h_i, U, R_l;
- * Algorithm 1, steps 6-12; Appendix A.2, "stored in sorted order and mapped to compact indices").
+ * Algorithm 1, steps 6-12; Appendix A.2: U is kept sorted and its members are numbered once per request).
  *
  *   h_i  = max{ l : i in S_l }  (-1 if i is in no S_l);   U = { i : h_i >= 0 } ascending;
  *   u_rank[i] = index of i in U (or -1);   R_l = { c : h_{U[c]} >= l } as ascending ranks c.
@@ -298,7 +298,7 @@ relaxkv_status relaxkv_mean_scores(const relaxkv_shape* shape, int32_t n_layers,
 
 /*
  * The user query's own attention at one layer with the context scores taken from the same pass (Section 2,
- * "running the query against the cached keys produces query-to-context attention at every layer"; Section 3.2, score
+ * the query's pass over the naive cache is what yields its attention to the context, layer by layer; Section 3.2, score
  * equation with the row normalisers of the query's real forward pass, whose softmax also spans the query's own
  * tokens).  For a serving caller this replaces relaxkv_score_select's scoring for the layer: the statistics pass
  * never runs, the scores come out of the forward pass the query makes anyway.
@@ -328,7 +328,7 @@ relaxkv_status relaxkv_scale_scores(const relaxkv_shape* shape, int32_t n_layers
 
 /*
  * ---- Dense block work of the active targets (Algorithm 1, steps 14, 16 and 20; Section 3.3 for the
- * position IDs).  The method runs "the unchanged Transformer block" on the |R_l| active rows only; these
+ * position IDs).  The method leaves the Transformer block as it is and runs it on the |R_l| active rows only; these
  * calls are that block for a Llama-style pre-norm decoder.  All tensors bf16, row-major, 16-byte aligned,
  * feature counts multiples of 8; fp32 arithmetic inside.  The caller owns every buffer. ----
  */

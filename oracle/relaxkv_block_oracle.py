@@ -1,6 +1,6 @@
 """fp64 numpy oracle of the dense per-row block work around the repair attention (Algorithm 1, steps 14, 16,
-20: "compute Q/K/V for the active repair targets", "the unchanged output projection, residual connections,
-normalization, and MLP"; Section 3.3: RoPE keeps the original global position IDs).
+20: the projections of the active repair targets, then the block's own output projection, residuals,
+normalisation and MLP, all unchanged; Section 3.3: RoPE keeps the original global position IDs).
 
 TEST INFRASTRUCTURE ONLY, like relaxkv_oracle: plain definitions of a Llama-style pre-norm decoder block
 (RMSNorm -> fused QKV projection -> rotary embedding on q and k -> [attention] -> output projection +

@@ -3,8 +3,8 @@
 // multiply-adds), so this is a plain streaming kernel, not the 128-row tensor-core GEMM: each warp owns two output
 // features (16 per block: a 5120-wide projection is 320 blocks, all resident at once), its lanes stride over K in
 // 16-byte pieces with eight independent weight loads in flight per lane, x stays in L1, and a shuffle tree sums the
-// lanes' partial dot products in a fixed order.  (Algorithm 1 runs "the unchanged
-// Transformer block"; after the repair loop the same block serves the decode step of the TTFT region.)
+// lanes' partial dot products in a fixed order.  (Algorithm 1 runs the model's
+// own block unchanged; after the repair loop the same block serves the decode step of the TTFT region.)
 #include "common.cuh"
 #include "gemv.cuh"
 

@@ -1,7 +1,7 @@
 """The user query's own forward pass and the first decode step over the context cache: what surrounds the repair
-loop in the paper's time-to-first-token region (Section 2: running the query against the cached keys yields the
-query-to-context attention of every layer; reproducibility appendix: the timed region ends with query prefill and
-first-token decode).  Call sequencing over torch buffers only; every operation runs in the CUDA kernels behind
+loop in the paper's time-to-first-token region (Section 2: the scores come from a pass of the query over the naive
+cache, one attention per layer; reproducibility appendix: query prefill and the first token's decode close the timed
+region).  Call sequencing over torch buffers only; every operation runs in the CUDA kernels behind
 `binding`.
 
 Per layer the query's rows run the decoder block: RMSNorm, Q/K/V projections, per-head Q/K norm where the model has
