@@ -3,6 +3,7 @@
 // asynchronous copies.
 #include "common.cuh"
 #include "kv_move.cuh"
+#include "sm100_ptx.cuh"
 
 namespace relaxkv {
 
@@ -32,36 +33,15 @@ __device__ __forceinline__ int warp_lower_bound(const int* __restrict__ a, int n
   return lo;
 }
 
-// ---- bulk-copy helpers: rows travel global -> shared -> global through the copy engine (this GPU's memory only, never
-// multicast), so no thread ever holds the data and one lane keeps many kilobytes in flight ------------------------------
-__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src_smem, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit_and_drain() {
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void bar_expect(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait (about 0.2 s): false if the copies never landed; the caller reports and skips its stores.
-__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < (1u << 22); ++it) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
+// Rows travel global -> shared -> global through the copy engine (bulk asynchronous copies, this GPU's memory only,
+// never multicast), so no thread ever holds the data and one lane keeps many kilobytes in flight.
+using namespace ptx;
+
+// After an expired wait the copies may still be in flight: give them time to land before the block's shared memory
+// goes away (bounded; the same grace period the tensor-core kernels take).
+__device__ __forceinline__ void grace_period() {
+  const uint64_t t0 = global_timer_ns();
+  while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
 }
 
 constexpr int kMoveWarps = 2;              // warps per block; every warp works on its own rows, no block-wide barrier
@@ -87,12 +67,12 @@ __device__ __forceinline__ void issue_row_loads(uint32_t dst, const uint16_t* k_
                                                 int head_dim, long long src_head_stride, uint32_t bar) {
   const uint32_t head_bytes = (uint32_t)head_dim * 2, row_bytes = head_bytes * n_kv_heads;
   if (src_head_stride == head_dim) {        // heads contiguous: one copy per tensor
-    bulk_g2s(dst, k_src, row_bytes, bar);
-    bulk_g2s(dst + row_bytes, v_src, row_bytes, bar);
+    bulk_load(dst, k_src, row_bytes, bar);
+    bulk_load(dst + row_bytes, v_src, row_bytes, bar);
   } else {
     for (int g = 0; g < n_kv_heads; ++g) {
-      bulk_g2s(dst + g * head_bytes, k_src + g * src_head_stride, head_bytes, bar);
-      bulk_g2s(dst + row_bytes + g * head_bytes, v_src + g * src_head_stride, head_bytes, bar);
+      bulk_load(dst + g * head_bytes, k_src + g * src_head_stride, head_bytes, bar);
+      bulk_load(dst + row_bytes + g * head_bytes, v_src + g * src_head_stride, head_bytes, bar);
     }
   }
 }
@@ -101,12 +81,12 @@ __device__ __forceinline__ void issue_row_stores(uint16_t* k_dst, uint16_t* v_ds
                                                  long long dst_head_stride) {
   const uint32_t head_bytes = (uint32_t)head_dim * 2, row_bytes = head_bytes * n_kv_heads;
   if (dst_head_stride == head_dim) {
-    bulk_s2g(k_dst, src, row_bytes);
-    bulk_s2g(v_dst, src + row_bytes, row_bytes);
+    bulk_store(k_dst, src, row_bytes);
+    bulk_store(v_dst, src + row_bytes, row_bytes);
   } else {
     for (int g = 0; g < n_kv_heads; ++g) {
-      bulk_s2g(k_dst + g * dst_head_stride, src + g * head_bytes, head_bytes);
-      bulk_s2g(v_dst + g * dst_head_stride, src + row_bytes + g * head_bytes, head_bytes);
+      bulk_store(k_dst + g * dst_head_stride, src + g * head_bytes, head_bytes);
+      bulk_store(v_dst + g * dst_head_stride, src + row_bytes + g * head_bytes, head_bytes);
     }
   }
 }
@@ -129,15 +109,16 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
   // call); n_new_rows: rows k_new / v_new hold.  An index past either is reported and the row zero-filled.
   extern __shared__ __align__(128) uint8_t stage[];          // [warp][row of the warp][K row | V row]
   __shared__ __align__(8) unsigned long long bars[kMoveWarps];
+  __shared__ volatile int gave_up[kMoveWarps];
   const int B = rt.n_req;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long x0 = ((long long)blockIdx.x * kMoveWarps + warp) * rows_per_warp;
   if (x0 >= ctx_rows) return;
-  const uint32_t bar = smem_addr(&bars[warp]);
-  if (lane == 0) bar_init(bar, 1);
+  const uint32_t bar = smem_u32(&bars[warp]);
+  if (lane == 0) { gave_up[warp] = 0; mbar_init(bar, 1); fence_barrier_init(); }
   const long long total = (mode == RELAXKV_CTX_UNION) ? (long long)__ldg(u_cu + B) : rt.ctx_cu[B];
   const uint32_t row_bytes = (uint32_t)n_kv_heads * head_dim * 2;
-  const uint32_t my_stage = smem_addr(stage) + (uint32_t)(warp * rows_per_warp + lane) * 2u * row_bytes;   // lanes < rows_per_warp
+  const uint32_t my_stage = smem_u32(stage) + (uint32_t)(warp * rows_per_warp + lane) * 2u * row_bytes;   // lanes < rows_per_warp
   int my_kind = 3;                             // lane rr keeps the source of row rr: 0 = cache, 1 = fresh, 2 = zero fill, 3 = skip
   long long my_off = 0;
   int prev_b = -1, rho_next = 0;               // the R list of request prev_b has been walked up to rho_next
@@ -214,7 +195,7 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
   // rows that are copied: how many bytes the warp's barrier has to see
   const unsigned copy_mask = __ballot_sync(0xffffffffu, lane < rows_per_warp && my_kind <= 1);
   __syncwarp();
-  if (lane == 0 && copy_mask) bar_expect(bar, (uint32_t)__popc(copy_mask) * 2u * row_bytes);
+  if (lane == 0 && copy_mask) mbar_expect_tx(bar, (uint32_t)__popc(copy_mask) * 2u * row_bytes);
   __syncwarp();
   if (lane < rows_per_warp) {
     if (my_kind == 0)
@@ -234,15 +215,16 @@ gather_ctx_kernel(ReqTable rt, int mode, int n_kv_heads, int head_dim,
   }
   if (copy_mask) {
     bool ok = true;
-    if (lane == 0) ok = bar_wait(bar, 0);
+    if (lane == 0) ok = mbar_wait(bar, 0, &gave_up[warp]);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (!ok) {
-      if (lane == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_GATHER, (int)x0, -1);
+      if (lane == 0) { report(st, RELAXKV_ERR_TIMEOUT, KID_GATHER, (int)x0, -1); grace_period(); }
+      __syncwarp();
     } else if (lane < rows_per_warp && my_kind <= 1) {
       const long long o = (x0 + lane) * n_kv_heads * head_dim;
       issue_row_stores(k_out + o, v_out + o, my_stage, n_kv_heads, head_dim, head_dim);
     }
-    if (lane < rows_per_warp) bulk_commit_and_drain();      // shared memory must outlive the copies that read it
+    if (lane < rows_per_warp) bulk_store_commit_and_drain();      // shared memory must outlive the copies that read it
   }
 }
 
@@ -259,14 +241,15 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
   // direct != 0: u_pos holds the targets' positions themselves (packed by r_cu); r_rank is not read
   extern __shared__ __align__(128) uint8_t stage[];          // [warp][row of the warp][K row | V row]
   __shared__ __align__(8) unsigned long long bars[kMoveWarps];
+  __shared__ volatile int gave_up[kMoveWarps];
   const int B = rt.n_req;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long y0 = ((long long)blockIdx.x * kMoveWarps + warp) * rows_per_warp;
   if (y0 >= rt.tile_cu[B]) return;             // rt.tile_cu = prefix of the host bounds on |R_{l,b}|
-  const uint32_t bar = smem_addr(&bars[warp]);
-  if (lane == 0) bar_init(bar, 1);
+  const uint32_t bar = smem_u32(&bars[warp]);
+  if (lane == 0) { gave_up[warp] = 0; mbar_init(bar, 1); fence_barrier_init(); }
   const uint32_t row_bytes = (uint32_t)n_kv_heads * head_dim * 2;
-  const uint32_t my_stage = smem_addr(stage) + (uint32_t)(warp * rows_per_warp + lane) * 2u * row_bytes;   // lanes < rows_per_warp
+  const uint32_t my_stage = smem_u32(stage) + (uint32_t)(warp * rows_per_warp + lane) * 2u * row_bytes;   // lanes < rows_per_warp
   long long d = -1, s = 0;
   if (lane < rows_per_warp) {
     const long long y = y0 + lane;
@@ -296,18 +279,19 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
   }
   const unsigned copy_mask = __ballot_sync(0xffffffffu, d >= 0);
   if (!copy_mask) return;
-  if (lane == 0) bar_expect(bar, (uint32_t)__popc(copy_mask) * 2u * row_bytes);
+  if (lane == 0) mbar_expect_tx(bar, (uint32_t)__popc(copy_mask) * 2u * row_bytes);
   __syncwarp();
   if (d >= 0) issue_row_loads(my_stage, k_new + s, v_new + s, n_kv_heads, head_dim, head_dim, bar);
   bool ok = true;
-  if (lane == 0) ok = bar_wait(bar, 0);
+  if (lane == 0) ok = mbar_wait(bar, 0, &gave_up[warp]);
   ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
   if (!ok) {
-    if (lane == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_SCATTER, (int)y0, -1);
+    if (lane == 0) { report(st, RELAXKV_ERR_TIMEOUT, KID_SCATTER, (int)y0, -1); grace_period(); }
+    __syncwarp();
   } else if (d >= 0) {
     issue_row_stores(cache_k + d, cache_v + d, my_stage, n_kv_heads, head_dim, head_stride);
   }
-  if (lane < rows_per_warp) bulk_commit_and_drain();
+  if (lane < rows_per_warp) bulk_store_commit_and_drain();
 }
 
 relaxkv_status launch_gather(const relaxkv_shape* shape, int mode, const relaxkv_cache_view* cache,
