@@ -35,7 +35,7 @@ def close(got: torch.Tensor, ref: np.ndarray, abs_floor: float):
 
 
 @pytest.mark.parametrize("M,N,K,res", [(300, 512, 320, False), (129, 264, 72, True), (1000, 1024, 2048, True), (1, 8, 8, False),
-                                       (257, 1280, 640, False), (5000, 2304, 1024, True)])
+                                       (257, 1280, 640, False), (5000, 2304, 1024, True), (2, 520, 1032, True), (4, 136, 264, False)])
 def test_linear(M, N, K, res):
     """Both GEMM kernels: SM pairs (256 x 256 tiles per cluster; here 129, 1000 and 5000 rows) and the single-block
     one the library picks when an odd, small number of 128-row tiles would leave half a cluster idle (300, 257, 1)."""
@@ -52,6 +52,40 @@ def _check_linear(M, N, K, res):
     ref = blk.linear(blk.f64(bits(x)), blk.f64(bits(w)), blk.f64(bits(r)) if res else None)
     close(y, ref, abs_floor=2e-3)
     torch.testing.assert_close(y.float(), (x.float() @ w.float().T + (r.float() if res else 0)), rtol=2e-2, atol=2e-2)
+
+
+def test_linear_at_the_benchmark_shapes():
+    """The projections at the sizes the repair loop runs them for the 32K Qwen3-14B-shaped stack: 18 000 active rows
+    through a 5120 -> 5120 projection with residual (SM pairs) and the fused gate/up projection of 5120 -> 2 x 17408 on
+    2 000 rows; 128 rows (the query's prefill) and one row (a decode token) through the same weights.  Sampled
+    rows against the oracle, every element against torch's fp32 matmul of the same bf16 inputs."""
+    rng = np.random.default_rng(2)
+    w = rnd(5120, 5120, scale=5120 ** -0.5, seed=71)
+    for M in (18000, 128, 1):
+        x, r = rnd(M, 5120, seed=72), rnd(M, 5120, seed=73)
+        y = torch.full((M, 5120), 7.0, dtype=torch.bfloat16, device="cuda")
+        B().relaxkv_linear(x, w, y, residual=r)
+        st, detail = B().relaxkv_read_device_status()
+        assert st == 0, (st, detail)
+        torch.testing.assert_close(y.float(), x.float() @ w.float().T + r.float(), rtol=2e-2, atol=3e-2)
+        rows = np.unique(rng.integers(0, M, size=min(M, 24)))
+        idx = torch.from_numpy(rows).cuda()
+        ref = blk.linear(blk.f64(bits(x[idx])), blk.f64(bits(w)), blk.f64(bits(r[idx])))
+        close(y[idx], ref, abs_floor=4e-3)
+    wgu = rnd(2 * 17408, 5120, scale=5120 ** -0.5, seed=74)
+    tiled = B().tile_gate_up(wgu)
+    for M in (2000, 128, 1):
+        x = rnd(M, 5120, seed=75)
+        out = torch.full((M, 17408), 7.0, dtype=torch.bfloat16, device="cuda")
+        B().relaxkv_linear_swiglu(x, tiled, out)
+        st, detail = B().relaxkv_read_device_status()
+        assert st == 0, (st, detail)
+        rows = np.unique(rng.integers(0, M, size=min(M, 12)))
+        idx = torch.from_numpy(rows).cuda()
+        ref = blk.swiglu(blk.linear(blk.f64(bits(x[idx])), blk.f64(bits(wgu)), None))
+        close(out[idx], ref, abs_floor=4e-3)
+        gu = x.float() @ wgu.float().T
+        torch.testing.assert_close(out.float(), torch.nn.functional.silu(gu[:, :17408]) * gu[:, 17408:], rtol=2e-2, atol=3e-2)
 
 
 def test_rmsnorm_rope_swiglu():

@@ -214,3 +214,80 @@ def test_whole_ragged_batch_of_eight_in_one_call():
             assert torch.equal(k2[pos], f.k_new[f.row_cu[b]:f.row_cu[b + 1]]) and torch.equal(v2[pos], f.v_new[f.row_cu[b]:f.row_cu[b + 1]])
             touched[pos] = True
         assert torch.equal(k2[~touched], case.k_cache[l][~touched]) and torch.equal(v2[~touched], case.v_cache[l][~touched])
+
+
+def test_controlled_configurations_at_32k_sampled_rows():
+    """The explicit-list entry points at the size the benchmark times them (32K context, Qwen3-14B heads): global
+    repair targets that need not lie in U (a top-m of a seeded score vector, context U), and a layer-wise sparse
+    context of |U| entries with the method's targets.  Random anchors (what is checked is the list path, not the
+    scoring); sampled target rows against the oracle's list attention, the cache update bit-exact."""
+    from oracle import relaxkv_oracle as orc
+    from paper_2609_33503_b200 import binding as B
+    T = 32768
+    w = inputs.qwen14b_32k("calibrated", 0.15, n_layers=2)
+    rng = np.random.default_rng(321)
+    k = [max(1, round(0.15 * T))]
+    override = [[np.sort(rng.choice(T, size=k[0], replace=False)).astype(np.int32)] for _ in range(2)]
+    case = Case(w, anchors_override=override)
+    s = case.make_session()
+    sets = case.sets[0]
+    n_u = len(sets.u_pos)
+    g = rng.random(T).astype(np.float32)
+    view = case.cache_views()[0]
+    cfgs = {"global_targets": (sets.u_pos.astype(np.int32), orc.topk(g.astype(np.float64), min(int(0.2 * T), n_u)).astype(np.int32)),
+            "layerwise_sparse": (orc.topk(rng.random(T), n_u).astype(np.int32), sets.positions(0).astype(np.int32))}
+    for name, (ctx, tgt) in cfgs.items():
+        q, kn, vn = inputs.fresh_qkv(w, 0, 0, case.k_cache[0], case.v_cache[0], torch.from_numpy(tgt.astype(np.int64)))
+        dev = case.device
+        ctx_pos, tgt_pos = torch.from_numpy(ctx).to(dev), torch.from_numpy(tgt).to(dev)
+        ctx_cu = torch.tensor([0, len(ctx)], dtype=torch.int32, device=dev)
+        tgt_cu = torch.tensor([0, len(tgt)], dtype=torch.int32, device=dev)
+        out = torch.zeros_like(q)
+        B.relaxkv_list_attention(s.shape, view, q, kn, vn, ctx_pos, ctx_cu, tgt_pos, tgt_cu, [len(tgt)], [len(ctx)], out, s.workspace)
+        st, detail = B.relaxkv_read_device_status()
+        assert st == 0, (name, st, detail)
+        rows = sampled_rows(len(tgt), 50, 16, seed=9)
+        ref, _ = orc.list_attention(case.req_k(0, 0), case.req_v(0, 0), inputs.bf16_bits(q), inputs.bf16_bits(kn), inputs.bf16_bits(vn),
+                                    ctx, tgt, case.scale, rows=rows)
+        mx, mean = attention_errors(out[torch.from_numpy(rows.astype(np.int64)).to(dev)], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (name, mx, mean)
+        k2, v2 = case.k_cache[0].clone(), case.v_cache[0].clone()
+        B.relaxkv_scatter_kv_lists(s.shape, B.CacheView(k2, v2, [0]), kn, vn, tgt_pos, tgt_cu, [len(tgt)])
+        pos = tgt_pos.long()
+        assert torch.equal(k2[pos], kn) and torch.equal(v2[pos], vn)
+        keep = torch.ones(T, dtype=torch.bool, device=dev)
+        keep[pos] = False
+        assert torch.equal(k2[keep], case.k_cache[0][keep]) and torch.equal(v2[keep], case.v_cache[0][keep])
+
+
+def test_query_prefill_attention_at_32k():
+    """relaxkv_query_prefill_attention at the benchmark's size: 128 query tokens behind a 32K context, Qwen3-14B heads
+    (the launch the time-to-first-token region makes per layer).  Every query row against the oracle's causal attention;
+    the emitted context scores against the oracle's supplied-normaliser scores in full."""
+    from oracle import relaxkv_oracle as orc
+    from paper_2609_33503_b200 import binding as B
+    w = inputs.qwen14b_32k("calibrated", 0.15, n_layers=1)
+    T, Qn, H, Hkv, D = 32768, 128, w.n_q_heads, w.n_kv_heads, w.head_dim
+    scale = D ** -0.5
+    q, k, v = inputs.layer_qkv(w, 0, 0, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(17)
+    k_all = torch.cat([k, torch.randn(Qn + 1, Hkv, D, device="cuda", generator=g).to(torch.bfloat16)]).contiguous()
+    v_all = torch.cat([v, torch.randn(Qn + 1, Hkv, D, device="cuda", generator=g).to(torch.bfloat16)]).contiguous()
+    shape = B.Shape(H, Hkv, D, [T], [Qn], scale)
+    ext = B.Shape(H, Hkv, D, [T + Qn], [Qn], scale)
+    ws = torch.empty(B.relaxkv_workspace_bytes(ext, 1) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.zeros_like(q)
+    lse = torch.zeros(H, Qn, dtype=torch.float32, device="cuda")
+    raw = torch.zeros(T, dtype=torch.float32, device="cuda")
+    B.relaxkv_query_prefill_attention(shape, B.CacheView(k_all, v_all, [0]), q, out, lse, raw, ws)
+    st, detail = B.relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+    kb, vb, qb = inputs.bf16_bits(k_all[:T + Qn]), inputs.bf16_bits(v_all[:T + Qn]), inputs.bf16_bits(q)
+    ref, ref_lse = orc.list_attention(kb, vb, qb, None, None, np.arange(T + Qn), np.arange(T, T + Qn), scale)
+    mx, mean = attention_errors(out, ref)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    np.testing.assert_allclose(lse.cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+    ref_raw = orc.raw_scores(qb, kb[:T], scale, lse=ref_lse.T)
+    got = raw.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - ref_raw) <= 1e-3 * ref_raw + 1e-6 / T), np.abs(got / ref_raw - 1).max()
