@@ -226,52 +226,59 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kBM, kBN, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
       bool ok = mbar_wait(bar_q, 0, abort_flag);
-      // S_x = Q_x K_j^T  -> bar_sfull[x]
-      auto issue_qk = [&](int x, int j) {
-        const int s = (2 * j) % kRing;
+      // This lane issues every MMA, and each instruction it executes in between delays the next one (measured: the
+      // step got 1 % shorter when the ring-slot and barrier arithmetic below replaced a modulo and a division per
+      // use).  So the positions are carried along and advanced once per step: ring slot of the step's V tile and of
+      // the K tile behind it, and the pair barrier (byte offset, phase) that covers the two.
+      uint32_t sv = 1, sk = 2, pk = 8, pph = 0;
+      const int n0 = n_my[0], n1 = n_my[1];
+      auto issue_qk = [&](int x, uint32_t slot) {                   // S_x = Q_x K^T with the K tile in `slot` -> bar_sfull[x]
         mma_ss_kloop<kHalves>(tmem_base + x * 128, desc_lo(q_smem + x * L::kTileBytes, 16),
-                              desc_lo(kv_smem + s * L::kTileBytes, 16), desc_hi_sw128(1024), idesc_qk);
+                              desc_lo(kv_smem + slot * L::kTileBytes, 16), desc_hi_sw128(1024), idesc_qk);
         mma_commit(bar_sfull + 8 * x);
       };
-      // O_x += P_x V_j   (P_x read from TMEM where the softmax warps left it, over S_x)
-      auto issue_pv = [&](int x, int j) -> bool {
-        const int s = (2 * j + 1) % kRing;
-        if (!mbar_wait(bar_pfull + 8 * x, j & 1, abort_flag)) return false;
+      // O_x += P_x V   (P_x read from TMEM where the softmax warps left it, over S_x; V in slot sv)
+      auto issue_pv = [&](int x, uint32_t par, uint32_t acc) -> bool {
+        const uint32_t v_lo = desc_lo(kv_smem + sv * L::kTileBytes, kHalfBytes);
+        if (!mbar_wait(bar_pfull + 8 * x, par, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t v_lo = desc_lo(kv_smem + s * L::kTileBytes, kHalfBytes);
-        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128, v_lo, desc_hi_sw128(1024), idesc_pv, j > 0 ? 1u : 0u);
+        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128, v_lo, desc_hi_sw128(1024), idesc_pv, acc);
         // the second half of P arrives while the first half is being multiplied
-        if (!mbar_wait(bar_pfull_hi + 8 * x, j & 1, abort_flag)) return false;
+        if (!mbar_wait(bar_pfull_hi + 8 * x, par, abort_flag)) return false;
         tc_fence_after();
         mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128 + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
-        if (j == n_my[x] - 1) mma_commit(bar_ofinal + 8 * x);
         return true;
       };
       // pair 0 = K_0 alone
       if (ok) ok = mbar_wait(bar_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        if (n_my[0] > 0) issue_qk(0, 0);
-        if (n_my[1] > 0) issue_qk(1, 0);
+        if (n0 > 0) issue_qk(0, 0);
+        if (n1 > 0) issue_qk(1, 0);
         mma_commit(bar_empty);
       }
       for (int j = 0; ok && j < n_my_max; ++j) {                // j counted from j0; this step consumes pair j + 1
-        const int pr = j + 1;
-        if (!(ok = mbar_wait(bar_full + 8 * (pr % L::kPairBars), (uint32_t)(pr / L::kPairBars) & 1, abort_flag))) break;
+        if (!(ok = mbar_wait(bar_full + pk, pph, abort_flag))) break;
         if (need_v_fix && j == v_fix_tile) {                    // V_j reaches past the request's end: have those rows zeroed
           mbar_arrive(bar_vreq);
           if (!(ok = mbar_wait(bar_vfix, 0, abort_flag))) break;
         }
         tc_fence_after();
-        if (j < n_my[0]) {
-          if (!(ok = issue_pv(0, j))) break;
-          if (j + 1 < n_my[0]) issue_qk(0, j + 1);
+        const uint32_t par = (uint32_t)j & 1u, acc = j > 0 ? 1u : 0u;
+        if (j < n0) {
+          if (!(ok = issue_pv(0, par, acc))) break;
+          if (j == n0 - 1) mma_commit(bar_ofinal);
+          if (j + 1 < n0) issue_qk(0, sk);
         }
-        if (j < n_my[1]) {
-          if (!(ok = issue_pv(1, j))) break;
-          if (j + 1 < n_my[1]) issue_qk(1, j + 1);
+        if (j < n1) {
+          if (!(ok = issue_pv(1, par, acc))) break;
+          if (j == n1 - 1) mma_commit(bar_ofinal + 8);
+          if (j + 1 < n1) issue_qk(1, sk);
         }
-        mma_commit(bar_empty + 8 * (pr % L::kPairBars));        // V_j and K_{j+1}: free once both tiles are through
+        mma_commit(bar_empty + pk);                             // V_j and K_{j+1}: free once both tiles are through
+        sv += 2; if (sv >= kRing) sv -= kRing;
+        sk += 2; if (sk >= kRing) sk -= kRing;
+        pk += 8; if (pk == 8 * L::kPairBars) { pk = 0; pph ^= 1u; }
       }
     }
   } else if (warp == 10 && need_v_fix) {
