@@ -70,6 +70,11 @@ typedef struct {
                                  /* blocks (up to 32, and as far as the workspace's 2048 row-splits allow) and merge   */
                                  /* the partial results by their log-sum-exp; automatic = only when the call has too   */
                                  /* few query tiles to fill the GPU (a query prefill, a decode step, few targets)      */
+  int32_t attention_persistent;  /* the repair / list attention calls have a persistent form (one thread block per SM  */
+                                 /* walks the call's query tiles, longest context first).  0: the library takes it     */
+                                 /* for one-split calls over gathered contexts of at most 128 key tiles; 1: for every  */
+                                 /* one-split call over a gathered context; 2: never.  Same results bit for bit.       */
+  int32_t attention_grid_blocks; /* > 0: number of thread blocks of the persistent form (default: one per SM)          */
 } relaxkv_tuning;
 
 /* Shapes shared by all calls. */

@@ -37,7 +37,8 @@ class RelaxKVError(RuntimeError):
 
 
 class _Tuning(ctypes.Structure):
-    _fields_ = [("attention_ctx_splits", ctypes.c_int32)]
+    _fields_ = [("attention_ctx_splits", ctypes.c_int32), ("attention_persistent", ctypes.c_int32),
+                ("attention_grid_blocks", ctypes.c_int32)]
 
 
 class _Shape(ctypes.Structure):
@@ -105,7 +106,7 @@ class Shape:
 
     def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, ctx_lens: Sequence[int],
                  q_lens: Optional[Sequence[int]] = None, softmax_scale: Optional[float] = None,
-                 attention_ctx_splits: int = 0):
+                 attention_ctx_splits: int = 0, attention_persistent: int = 0, attention_grid_blocks: int = 0):
         self.ctx_lens = [int(x) for x in ctx_lens]
         self.q_lens = None if q_lens is None else [int(x) for x in q_lens]
         self._ctx = _i32(self.ctx_lens)
@@ -117,12 +118,12 @@ class Shape:
         self.c.h_q_len = ctypes.cast(self._q, ctypes.POINTER(ctypes.c_int32)) if self._q is not None else None
         self.c.softmax_scale = float(softmax_scale if softmax_scale is not None else head_dim ** -0.5)
         self._tuning = None
-        self.set_tuning(attention_ctx_splits)
+        self.set_tuning(attention_ctx_splits, attention_persistent, attention_grid_blocks)
 
-    def set_tuning(self, attention_ctx_splits: int = 0) -> None:
+    def set_tuning(self, attention_ctx_splits: int = 0, attention_persistent: int = 0, attention_grid_blocks: int = 0) -> None:
         """relaxkv_tuning of the calls made with this shape (0 = the library's automatic choice)."""
-        if attention_ctx_splits:
-            self._tuning = _Tuning(int(attention_ctx_splits))
+        if attention_ctx_splits or attention_persistent or attention_grid_blocks:
+            self._tuning = _Tuning(int(attention_ctx_splits), int(attention_persistent), int(attention_grid_blocks))
             self.c.h_tuning = ctypes.pointer(self._tuning)
         else:
             self._tuning = None

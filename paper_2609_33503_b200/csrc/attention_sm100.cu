@@ -35,6 +35,7 @@ constexpr int kBM = 128;                      // query rows per tile (TMEM lanes
 constexpr int kBN = 128;                      // keys per context tile
 constexpr int kHalfBytes = 128 * 128;         // 128 rows x 64 bf16: one 128B-swizzled half tile
 constexpr int kRing = 5;                      // K/V tile buffers, used in the order K0 V0 K1 V1 ...
+constexpr int kPersistMaxTiles = 128;          // contexts up to this many key tiles take the persistent form
 constexpr int kAttnThreads = 384;             // 2 x 4 softmax warps + a control warpgroup (TMA warp, MMA warp, 2 idle)
 
 template <int D>
@@ -50,6 +51,93 @@ struct AttnSmem {
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                // slack to align the base to 1024 B
 };
+
+// One step of a query row's online softmax (thread = query row = TMEM lane): S_x(j) is read from TMEM, the keys
+// past the row's limit are masked on the tiles that straddle the staircase (col0 = index of the tile's first key),
+// the running maximum m and sum z are updated (O_x is rescaled only when the maximum grew by more than the
+// threshold), and P is written over S as bf16 in two column halves, each handed to the MMA warp (bar_p_lo,
+// bar_p_hi) as soon as it is stored.
+template <int D>
+__device__ __forceinline__ void softmax_step(uint32_t t_s, uint32_t t_o, int col0, int limit, bool first, float scale_log2,
+                                             float& m, float& z, uint32_t bar_p_lo, uint32_t bar_p_hi) {
+  uint32_t s[kBN];
+#pragma unroll
+  for (int c = 0; c < kBN / 32; ++c) tmem_ld32(t_s + c * 32, &s[c * 32]);
+  tmem_wait_ld();
+  if (col0 + kBN - 1 > limit) {
+#pragma unroll
+    for (int i = 0; i < kBN; ++i)
+      if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
+  }
+  // row maximum: eight independent chains instead of one 128-deep dependency chain
+  float mx8[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
+#pragma unroll
+  for (int i = 8; i + 16 <= kBN; i += 16) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mx8[e] = fmax3(mx8[e], __uint_as_float(s[i + e]), __uint_as_float(s[i + 8 + e]));
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[kBN - 8 + e]));
+  const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                         fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+  const float m_new = mx * scale_log2;
+  if (first) {
+    m = fmaxf(m_new, -1.0e30f);           // a row whose first tile of this split is fully masked keeps a finite reference
+  } else {
+    // S_x(j) is complete, hence so is O_x += P_x V_{j-1}: O_x may be rescaled here
+    const bool need = m_new > m + kRescaleThreshold;
+    if (__any_sync(0xffffffffu, need)) {
+      float alpha = 1.f;
+      if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(t_o + c * 32, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+        tmem_st32(t_o + c * 32, o);
+      }
+      tmem_wait_st();
+    }
+  }
+  float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
+  const float neg_m = -m;
+#pragma unroll
+  for (int c = 0; c < kBN / 32; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+      // p = 2^(s * scale - m) for eight keys; the scaling and the row sums use packed fp32 pairs
+      float x[8], p[8];
+#pragma unroll
+      for (int e = 0; e < 8; e += 2)
+        fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
+             scale_log2, neg_m, neg_m);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
+      add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
+      add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
+#pragma unroll
+      for (int e = 0; e < 8; e += 2) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(p[e], p[e + 1]);
+        pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h);
+      }
+    }
+    tmem_st16(t_s + c * 16, pk);
+    if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p_lo);
+    }
+  }
+  z += (zs0 + zs1) + (zs2 + zs3);
+  tmem_wait_st();
+  tc_fence_before();
+  mbar_arrive(bar_p_hi);
+}
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -326,84 +414,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[kBN];
-#pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) tmem_ld32(t_s + c * 32, &s[c * 32]);
-      tmem_wait_ld();
-      const int col0 = (j0 + j) * kBN;
-      if (col0 + kBN - 1 > limit) {
-#pragma unroll
-        for (int i = 0; i < kBN; ++i)
-          if (col0 + i > limit) s[i] = 0xff800000u;              // -inf
-      }
-      // row maximum: eight independent chains instead of one 128-deep dependency chain
-      float mx8[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[e]);
-#pragma unroll
-      for (int i = 8; i + 16 <= kBN; i += 16) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) mx8[e] = fmax3(mx8[e], __uint_as_float(s[i + e]), __uint_as_float(s[i + 8 + e]));
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(s[kBN - 8 + e]));
-      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-      const float m_new = mx * scale_log2;
-      if (j == 0) {
-        m = fmaxf(m_new, -1.0e30f);           // a row whose first tile of this split is fully masked keeps a finite reference
-      } else {
-        // S_x(j) is complete, hence so is O_x += P_x V_{j-1}: O_x may be rescaled here
-        const bool need = m_new > m + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          float alpha = 1.f;
-          if (need) { alpha = fast_exp2(m - m_new); z *= alpha; m = m_new; }
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(t_o + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st32(t_o + c * 32, o);
-          }
-          tmem_wait_st();
-        }
-      }
-      float zs0 = 0.f, zs1 = 0.f, zs2 = 0.f, zs3 = 0.f;
-      const float neg_m = -m;
-#pragma unroll
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          // p = 2^(s * scale - m) for eight keys; the scaling and the row sums use packed fp32 pairs
-          float x[8], p[8];
-#pragma unroll
-          for (int e = 0; e < 8; e += 2)
-            fma2(x[e], x[e + 1], __uint_as_float(s[c * 32 + i + e]), __uint_as_float(s[c * 32 + i + e + 1]), scale_log2,
-                 scale_log2, neg_m, neg_m);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) p[e] = fast_exp2(x[e]);
-          add2(zs0, zs1, p[0], p[1]); add2(zs2, zs3, p[2], p[3]);
-          add2(zs0, zs1, p[4], p[5]); add2(zs2, zs3, p[6], p[7]);
-#pragma unroll
-          for (int e = 0; e < 8; e += 2) {
-            __nv_bfloat162 h = __floats2bfloat162_rn(p[e], p[e + 1]);
-            pk[(i + e) >> 1] = *reinterpret_cast<uint32_t*>(&h);
-          }
-        }
-        tmem_st16(t_s + c * 16, pk);
-        if (c == kBN / 64 - 1) {          // first 64 keys done: hand them to the MMA warp early
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(my_pfull);
-        }
-      }
-      z += (zs0 + zs1) + (zs2 + zs3);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_pfull_hi + 8 * x);
+      softmax_step<D>(t_s, t_o, (j0 + j) * kBN, limit, j == 0, scale_log2, m, z, my_pfull, bar_pfull_hi + 8 * x);
     }
     if (ok && my_n > 0) {
       ok = mbar_wait(bar_ofinal + 8 * x, 0, abort_flag);
@@ -477,6 +488,495 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// Persistent form of the kernel above, for calls whose blocks are short (a context of at most 128 tiles): one block
+// per SM walks work items (pair of query tiles x KV head, the same list in the same longest-first order) that its
+// producer lane claims from a global counter a few steps before the current item ends.  Barriers, tensor memory and
+// the K/V ring live across items; the next item's first K tile travels with the current item's last V tile, its Q
+// tiles are loaded as soon as the current item's last Q K^T has completed, and its first Q K^T is issued right behind
+// the current item's last P V, so a block turn-over costs about 5 k clk instead of about 14 k.  Items reach the other
+// roles as 64-byte records in a two-slot mailbox in shared memory.  One split only, gathered contexts only (the
+// cache-only calls keep the kernel above).  Same arithmetic per row, hence the same bits.
+// ---------------------------------------------------------------------------------------------------------------------
+template <int D>
+struct PersistSmem {
+  static constexpr int kHalves = D / 64;
+  static constexpr int kTileBytes = kHalves * kHalfBytes;
+  static constexpr int kQ = 0;
+  static constexpr int kKV = kQ + 2 * kTileBytes;
+  static constexpr int kBar = kKV + kRing * kTileBytes;
+  static constexpr int kPairBars = 3;
+  // q | s, p, p_hi, ofinal x2 | pairs full/empty | qfree | odrained x2 | item full x2 | item free x2
+  static constexpr int kNumBars = 1 + 8 + 2 * kPairBars + 1 + 2 + 2 + 2;
+  static constexpr int kMisc = kBar + 8 * kNumBars;                     // tmem address, abort flag, two item records
+  static constexpr int kTotal = kMisc + 8 + 2 * 64;
+  static constexpr int kDynamic = kTotal + 1024;
+};
+
+// One work item as every role needs it; 16 ints so that it travels through shared memory as four 16-byte pieces.
+struct WorkItem {
+  int work;            // 1: work, -1: the list is exhausted
+  int n_max, n_my0, n_my1;
+  int n_valid0, n_valid1, hd, q_row_base;
+  int nu, ctx_len_b, r_base, rho0;      // r_base = r_cu[b]
+  int u_base, ctx_base, b, pad;         // u_base = u_cu[b]
+  __device__ __forceinline__ int n_valid(int x) const { return x ? n_valid1 : n_valid0; }
+  __device__ __forceinline__ int n_my(int x) const { return x ? n_my1 : n_my0; }
+};
+__device__ __forceinline__ void item_store(int4* rec, const WorkItem& it) {
+  rec[0] = make_int4(it.work, it.n_max, it.n_my0, it.n_my1);
+  rec[1] = make_int4(it.n_valid0, it.n_valid1, it.hd, it.q_row_base);
+  rec[2] = make_int4(it.nu, it.ctx_len_b, it.r_base, it.rho0);
+  rec[3] = make_int4(it.u_base, it.ctx_base, it.b, 0);
+}
+__device__ __forceinline__ void item_load_head(const int4* rec, WorkItem& it) {      // what the MMA issuer needs
+  const int4 a = rec[0];
+  it.work = a.x; it.n_max = a.y; it.n_my0 = a.z; it.n_my1 = a.w;
+}
+__device__ __forceinline__ void item_load(const int4* rec, WorkItem& it) {
+  item_load_head(rec, it);
+  const int4 b = rec[1], c = rec[2], d = rec[3];
+  it.n_valid0 = b.x; it.n_valid1 = b.y; it.hd = b.z; it.q_row_base = b.w;
+  it.nu = c.x; it.ctx_len_b = c.y; it.r_base = c.z; it.rho0 = c.w;
+  it.u_base = d.x; it.ctx_base = d.y; it.b = d.z; it.pad = 0;
+}
+
+__device__ __forceinline__ WorkItem decode_item(int id, const ReqTable& rt, int head_inner, int Hkv, int mode, int tile_targets,
+                                                const int* __restrict__ u_pos, const int* __restrict__ u_cu,
+                                                const int* __restrict__ r_rank, const int* __restrict__ r_cu,
+                                                long long n_target_rows, DeviceStatus* st) {
+  WorkItem it;
+  it.work = 0; it.pad = 0;
+  const int B = rt.n_req;
+  const int n_pairs_total = rt.tile_cu[B];
+  it.hd = head_inner ? (id % Hkv) : (id / n_pairs_total);
+  const int tt = head_inner ? (id / Hkv) : (id - it.hd * n_pairs_total);
+  const int b = find_segment(rt.tile_cu, B, tt);
+  it.b = b;
+  const int p_rev = tt - rt.tile_cu[b];
+  it.r_base = r_cu[b]; it.u_base = u_cu[b];
+  const int nr = r_cu[b + 1] - it.r_base;
+  const int nu = u_cu[b + 1] - it.u_base;
+  it.nu = nu;
+  const int pair_targets = 2 * tile_targets;
+  const int n_pairs_true = (nr + pair_targets - 1) / pair_targets;
+  it.n_max = 0; it.n_my0 = it.n_my1 = 0; it.n_valid0 = it.n_valid1 = 0;
+  it.rho0 = 0; it.ctx_len_b = 0; it.ctx_base = 0; it.q_row_base = 0;
+  if (p_rev >= n_pairs_true) return it;
+  if (nr > rt.bound_a[b] || (mode == RELAXKV_CTX_UNION && nu > rt.bound_b[b]) || (long long)(r_cu[b + 1] - r_cu[0]) > n_target_rows) {
+    report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, nr, nu);
+    return it;
+  }
+  const int pair = n_pairs_true - 1 - p_rev;
+  it.rho0 = pair * pair_targets;
+  it.ctx_len_b = (mode == RELAXKV_CTX_UNION) ? nu : rt.ctx_len[b];
+  it.ctx_base = (int)((mode == RELAXKV_CTX_UNION) ? (long long)it.u_base : rt.ctx_cu[b]);
+  it.q_row_base = (it.r_base - r_cu[0]) + it.rho0;
+  int nm[2] = {0, 0}, nv[2] = {0, 0};
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    nv[x] = max(0, min(tile_targets, nr - it.rho0 - x * tile_targets));
+    if (nv[x] > 0) {
+      const int c = r_rank[it.r_base + it.rho0 + x * tile_targets + nv[x] - 1];
+      const int cc = min(max(c, 0), max(nu - 1, 0));
+      int lim_last = (mode == RELAXKV_CTX_UNION) ? cc : u_pos[it.u_base + cc];
+      lim_last = min(max(lim_last, 0), it.ctx_len_b - 1);
+      nm[x] = lim_last / kBN + 1;
+    }
+  }
+  it.n_valid0 = nv[0]; it.n_valid1 = nv[1]; it.n_my0 = nm[0]; it.n_my1 = nm[1];
+  it.n_max = max(nm[0], nm[1]);
+  it.work = it.n_max > 0;
+  return it;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_persist_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                         const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ ReqTable rt,
+                         int mode, int allow_empty, int head_inner, int H, int Hkv, int tile_targets, float scale_log2,
+                         const int* __restrict__ u_pos, const int* __restrict__ u_cu,
+                         const int* __restrict__ r_rank, const int* __restrict__ r_cu,
+                         long long n_target_rows, uint16_t* __restrict__ out, float* __restrict__ lse_out,
+                         int total_items, int* __restrict__ work_counter, DeviceStatus* st) {
+  using L = PersistSmem<D>;
+  constexpr int kHalves = L::kHalves;
+  constexpr uint32_t kTmemCols = 512;
+  const int G = H / Hkv;
+  if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_smem = base + L::kQ, kv_smem = base + L::kKV;
+  const uint32_t bar0 = base + L::kBar;
+  const uint32_t bar_q = bar0;
+  const uint32_t bar_sfull = bar0 + 8, bar_pfull = bar0 + 24, bar_pfull_hi = bar0 + 40, bar_ofinal = bar0 + 56;
+  const uint32_t bar_full = bar0 + 72, bar_empty = bar_full + 8 * L::kPairBars;
+  const uint32_t bar_qfree = bar_empty + 8 * L::kPairBars;
+  const uint32_t bar_odrained = bar_qfree + 8;          // [2]
+  const uint32_t bar_item = bar_odrained + 16;          // [2]
+  const uint32_t bar_itemfree = bar_item + 16;          // [2]
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kMisc + 4);
+  int4* item_rec = reinterpret_cast<int4*>(base_ptr + L::kMisc + 8 + 8);   // two records of 64 bytes, 16-byte aligned
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull + 8 * x, 1); mbar_init(bar_pfull + 8 * x, 128); mbar_init(bar_pfull_hi + 8 * x, 128); mbar_init(bar_ofinal + 8 * x, 1); }
+    for (int s = 0; s < L::kPairBars; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_qfree, 1);
+    for (int x = 0; x < 2; ++x) { mbar_init(bar_odrained + 8 * x, 128); mbar_init(bar_item + 8 * x, 1); mbar_init(bar_itemfree + 8 * x, 2 * kBM + 1); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 9) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols); tmem_relinquish(); }
+  {
+    const int used = tile_targets * G;
+    const int n_pad = kBM - used;
+    for (int i = threadIdx.x; i < n_pad * 8 * kHalves * 2; i += kAttnThreads) {
+      const int piece = i & 7, r = (i >> 3) % n_pad, blk = (i >> 3) / n_pad;
+      *reinterpret_cast<uint4*>(base_ptr + L::kQ + blk * kHalfBytes + (used + r) * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // The k-th published record sits in slot k & 1 (phase k >> 1).  A reader copies it and arrives on the slot's
+  // "free" barrier; the producer overwrites a slot only after all 257 readers of its previous record have done so.
+  auto read_item = [&](int k, WorkItem& it, bool head_only) -> bool {
+    if (!mbar_wait(bar_item + 8 * (k & 1), (uint32_t)(k >> 1) & 1, abort_flag)) return false;
+    if (head_only) item_load_head(item_rec + 4 * (k & 1), it); else item_load(item_rec + 4 * (k & 1), it);
+    mbar_arrive(bar_itemfree + 8 * (k & 1));
+    return true;
+  };
+
+  if (warp >= 8) {
+  reg_dealloc<56>();
+  if (warp == 8) {
+    // ================= producer: work items, Q tiles, K/V tiles =================
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+      int n_fetched = 0, n_pub = 0;
+      bool ok = true;
+      auto fetch_work = [&](WorkItem& it) -> bool {          // next item that has work; false when the list is exhausted
+        for (;;) {
+          const int id = (n_fetched == 0) ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(work_counter, 1);
+          ++n_fetched;
+          if (id >= total_items) { it.work = -1; return false; }
+          it = decode_item(id, rt, head_inner, Hkv, mode, tile_targets, u_pos, u_cu, r_rank, r_cu, n_target_rows, st);
+          if (it.work) return true;
+        }
+      };
+      auto publish = [&](const WorkItem& it) -> bool {
+        const int k = n_pub;
+        if (k >= 2 && !mbar_wait(bar_itemfree + 8 * (k & 1), (uint32_t)((k - 2) >> 1) & 1, abort_flag)) return false;
+        item_store(item_rec + 4 * (k & 1), it);
+        mbar_arrive(bar_item + 8 * (k & 1));
+        ++n_pub;
+        return true;
+      };
+      auto load_q = [&](const WorkItem& it) {
+        mbar_expect_tx(bar_q, (uint32_t)(2 * kHalves * tile_targets * G * 128));
+        for (int x = 0; x < 2; ++x)
+          for (int hf = 0; hf < kHalves; ++hf)
+            tma_load_3d(q_smem + (x * kHalves + hf) * kHalfBytes, &tm_q, bar_q, hf * 64, it.hd * G, it.q_row_base + x * tile_targets);
+      };
+      auto load_tile = [&](int u, const WorkItem& it, int j, uint32_t bar) {      // u = 2 g for K of global tile g, 2 g + 1 for V
+        const int s = u % kRing;
+        const int row = it.ctx_base + j * kBN;
+        const CUtensorMap* tm = (u & 1) ? &tm_v : &tm_k;
+        for (int hf = 0; hf < kHalves; ++hf) tma_load_3d(kv_smem + s * L::kTileBytes + hf * kHalfBytes, tm, bar, hf * 64, it.hd, row);
+      };
+      WorkItem cur, nxt;
+      fetch_work(cur);
+      ok = publish(cur);
+      if (ok && cur.work > 0) {
+        load_q(cur);
+        int Gt = 0;                                                  // tile index, counted over the items, of cur's tile 0
+        int cw = 0;                                                  // work items done so far
+        for (;;) {
+          bool have_nxt = false, fetched = false;
+          for (int j = 0; ok && j <= cur.n_max; ++j) {               // pair g = (V_{g-1}, K_g)
+            if (!fetched && j >= cur.n_max - 2) {                    // claim the next item late (the list balances the SMs
+                                                                     // only if nobody holds work long before starting it),
+                                                                     // yet a few steps before the readers ask for it
+              have_nxt = fetch_work(nxt);
+              fetched = true;
+              if (!(ok = publish(nxt))) break;
+            }
+            if (j == 0 && cw > 0) continue;                          // loaded as the trailing pair of the previous item
+            const int g = Gt + j;
+            const bool has_v = j > 0;
+            const bool has_k = (j < cur.n_max) || have_nxt;
+            if (!has_v && !has_k) continue;
+            const uint32_t bar = bar_full + 8 * (uint32_t)(g % L::kPairBars);
+            if (g >= 3 && !(ok = mbar_wait(bar_empty + 8 * (uint32_t)((g - 3) % L::kPairBars), (uint32_t)((g - 3) / L::kPairBars) & 1, abort_flag))) break;
+            mbar_expect_tx(bar, (uint32_t)((has_v ? L::kTileBytes : 0) + (has_k ? L::kTileBytes : 0)));
+            if (has_v) load_tile(2 * g - 1, cur, j - 1, bar);
+            if (has_k) {
+              if (g >= 3 && !(ok = mbar_wait(bar_empty + 8 * (uint32_t)((g - 2) % L::kPairBars), (uint32_t)((g - 2) / L::kPairBars) & 1, abort_flag))) break;
+              if (j < cur.n_max) load_tile(2 * g, cur, j, bar); else load_tile(2 * g, nxt, 0, bar);
+            }
+          }
+          if (!ok || !have_nxt) break;
+          // every Q K^T of cur has completed: the Q tiles may be replaced
+          if (!(ok = mbar_wait(bar_qfree, (uint32_t)cw & 1, abort_flag))) break;
+          load_q(nxt);
+          Gt += cur.n_max; cur = nxt; ++cw;
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ================= MMA issuer =================
+    // One lane issues every MMA; each of its instructions delays the next one, so the loop over an item's inner steps
+    // holds nothing but the waits and the issues, and the item's first and last step (which also look at the previous
+    // item's epilogue and at the next item) run through a separate, general copy of the step.
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(kBM, kBN, 0);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(kBM, D, 1);
+      bool ok = true;
+      uint32_t k = 0;                       // index of the current item
+      uint32_t sp0 = 0, sp1 = 0;            // parity of each tile's next P (its S / P barriers complete once per step)
+      uint32_t op0 = 0, op1 = 0;            // epilogues of each tile so far (parity of its "O drained" barrier)
+      // running positions, advanced once per step: ring slot of the step's V tile and of the K tile behind it, and the
+      // pair barrier (offset, phase) that covers the two
+      uint32_t sv = 1, sk = 2, pk = 8;
+      uint32_t pph = 0;
+      auto issue_qk = [&](int x, uint32_t slot) {                   // S_x = Q_x K^T with the K tile in `slot`
+        mma_ss_kloop<kHalves>(tmem_base + x * 128, desc_lo(q_smem + x * L::kTileBytes, 16), desc_lo(kv_smem + slot * L::kTileBytes, 16),
+                              desc_hi_sw128(1024), idesc_qk);
+        mma_commit(bar_sfull + 8 * x);
+      };
+      auto issue_pv = [&](int x, uint32_t par, uint32_t acc) -> bool {   // O_x (+)= P_x V with the V tile in slot sv
+        const uint32_t v_lo = desc_lo(kv_smem + sv * L::kTileBytes, kHalfBytes);
+        if (!mbar_wait(bar_pfull + 8 * x, par, abort_flag)) return false;
+        tc_fence_after();
+        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128, v_lo, desc_hi_sw128(1024), idesc_pv, acc);
+        if (!mbar_wait(bar_pfull_hi + 8 * x, par, abort_flag)) return false;
+        tc_fence_after();
+        mma_ts_4steps(tmem_base + 256 + x * 128, tmem_base + x * 128 + 32, v_lo + 512, desc_hi_sw128(1024), idesc_pv, 1u);
+        return true;
+      };
+      auto advance = [&]() {
+        mma_commit(bar_empty + pk);
+        sv += 2; if (sv >= kRing) sv -= kRing;
+        sk += 2; if (sk >= kRing) sk -= kRing;
+        pk += 8; if (pk == 8 * L::kPairBars) { pk = 0; pph ^= 1u; }
+      };
+      WorkItem cur, nxt;
+      cur.work = 0; nxt.work = 0; nxt.n_max = nxt.n_my0 = nxt.n_my1 = 0;
+      ok = read_item(0, cur, true);
+      if (ok && cur.work > 0) {
+        ok = mbar_wait(bar_q, 0, abort_flag);
+        if (ok) ok = mbar_wait(bar_full, 0, abort_flag);
+        if (ok) {
+          tc_fence_after();
+          if (cur.n_my0 > 0) issue_qk(0, 0);
+          if (cur.n_my1 > 0) issue_qk(1, 0);
+          if (cur.n_max == 1) mma_commit(bar_qfree);
+          mma_commit(bar_empty);
+        }
+        while (ok) {
+          const int n0 = cur.n_my0, n1 = cur.n_my1, n_max = cur.n_max;
+          bool have_nxt = false;
+          // the general step: j = 0 and j = n_max - 1
+          auto edge_step = [&](int j) -> bool {
+            if (!mbar_wait(bar_full + pk, pph, abort_flag)) return false;
+            const bool last = (j == n_max - 1);
+            if (last) {                                             // the next item's record: shown early in cur
+              if (!read_item((int)k + 1, nxt, true)) return false;
+              have_nxt = nxt.work > 0;
+            }
+            tc_fence_after();
+            bool q_ready = false;
+            if (j < n0) {
+              if (j == 0 && op0 > 0) {                              // O_0 of the previous item must have been read out
+                if (!mbar_wait(bar_odrained, (op0 - 1) & 1u, abort_flag)) return false;
+                tc_fence_after();
+              }
+              if (!issue_pv(0, (sp0 + (uint32_t)j) & 1u, j > 0 ? 1u : 0u)) return false;
+              if (j == n0 - 1) mma_commit(bar_ofinal);
+              if (j + 1 < n0) issue_qk(0, sk);
+            }
+            if (last && have_nxt && mbar_try_wait(bar_q, (k + 1) & 1u)) {   // the next item's Q tiles have landed already
+              q_ready = true;
+              tc_fence_after();
+              if (nxt.n_my0 > 0) issue_qk(0, sk);
+            }
+            if (j < n1) {
+              if (j == 0 && op1 > 0) {
+                if (!mbar_wait(bar_odrained + 8, (op1 - 1) & 1u, abort_flag)) return false;
+                tc_fence_after();
+              }
+              if (!issue_pv(1, (sp1 + (uint32_t)j) & 1u, j > 0 ? 1u : 0u)) return false;
+              if (j == n1 - 1) mma_commit(bar_ofinal + 8);
+              if (j + 1 < n1) issue_qk(1, sk);
+            }
+            if (last && have_nxt) {
+              if (!q_ready) {
+                if (!mbar_wait(bar_q, (k + 1) & 1u, abort_flag)) return false;
+                tc_fence_after();
+                if (nxt.n_my0 > 0) issue_qk(0, sk);
+              }
+              if (nxt.n_my1 > 0) issue_qk(1, sk);
+              if (nxt.n_max == 1) mma_commit(bar_qfree);
+            }
+            advance();
+            return true;
+          };
+          if (!(ok = edge_step(0))) break;
+          // inner steps 1 .. n_max - 2
+          for (int j = 1; j < n_max - 1; ++j) {
+            if (!(ok = mbar_wait(bar_full + pk, pph, abort_flag))) break;
+            tc_fence_after();
+            if (j < n0) {
+              if (!(ok = issue_pv(0, (sp0 + (uint32_t)j) & 1u, 1u))) break;
+              if (j == n0 - 1) mma_commit(bar_ofinal);
+              if (j + 1 < n0) issue_qk(0, sk);
+            }
+            if (j < n1) {
+              if (!(ok = issue_pv(1, (sp1 + (uint32_t)j) & 1u, 1u))) break;
+              if (j == n1 - 1) mma_commit(bar_ofinal + 8);
+              if (j + 1 < n1) issue_qk(1, sk);
+            }
+            advance();
+          }
+          if (!ok) break;
+          if (n_max >= 2) {
+            mma_commit(bar_qfree);                                  // the last Q K^T of cur has been issued
+            if (!(ok = edge_step(n_max - 1))) break;
+          }
+          sp0 += (uint32_t)n0; sp1 += (uint32_t)n1;
+          op0 += (n0 > 0) ? 1u : 0u; op1 += (n1 > 0) ? 1u : 0u;
+          if (!have_nxt) break;
+          cur = nxt; ++k;
+        }
+      }
+    }
+  }
+  } else {
+    reg_alloc<224>();
+    // ================= softmax + epilogue =================
+    const int x = warp >> 2;
+    const int row = threadIdx.x & 127;
+    const int t_local = row / G, j_head = row - t_local * G;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_s = lane_base + x * 128, t_o = lane_base + 256 + x * 128;
+    const uint32_t my_sfull = bar_sfull + 8 * x, my_pfull = bar_pfull + 8 * x;
+    const uint32_t rec_smem = smem_u32(item_rec);
+    // One register of phase state: bit 0 = parity of this tile's next S, bit 1 = parity of its next final O,
+    // bits 2.. = index of the current item.  The item's record stays in shared memory (its slot is released only
+    // after the epilogue), so that little of it has to live in registers across the key loop.
+    uint32_t ph = 0;
+    auto rec_ld = [&](uint32_t k, int piece) -> int4 {
+      int4 v;
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(rec_smem + (k & 1u) * 64u + piece * 16u));
+      return v;
+    };
+    auto wait_rec = [&](uint32_t k) -> bool { return mbar_wait(bar_item + 8 * (k & 1u), (k >> 1) & 1u, abort_flag); };
+    // this thread's row of item k: validity and the load of its context rank
+    auto row_rank = [&](uint32_t k, bool& valid) -> int {
+      const int4 a = rec_ld(k, 0), b = rec_ld(k, 1), cc = rec_ld(k, 2);
+      valid = a.x > 0 && (row < tile_targets * G) && (t_local < (x ? b.y : b.x));
+      return valid ? r_rank[cc.z + cc.w + x * tile_targets + t_local] : 0;
+    };
+    bool ok = wait_rec(0);
+    bool row_valid = false;
+    int c = ok ? row_rank(0, row_valid) : 0;
+    while (ok) {
+      const uint32_t k = ph >> 2;
+      int limit = 0, my_n;
+      bool row_empty = false;
+      {
+        const int4 a = rec_ld(k, 0);
+        if (a.x <= 0) { mbar_arrive(bar_itemfree + 8 * (k & 1u)); break; }
+        my_n = x ? a.w : a.z;
+        if (row_valid) {
+          const int4 cc = rec_ld(k, 2), d = rec_ld(k, 3);
+          const int nu = cc.x, ctx_len_b = cc.y;
+          if (c == -1 && allow_empty) {
+            row_empty = true;
+          } else if (c < 0 || c >= nu) {
+            report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, c, nu);
+          } else {
+            limit = (mode == RELAXKV_CTX_UNION) ? c : u_pos[d.x + c];
+            if (limit < 0 || limit >= ctx_len_b) { report(st, RELAXKV_ERR_BAD_INDEX, KID_ATTN_SM100, limit, ctx_len_b); limit = 0; }
+          }
+        }
+      }
+      float m = -INFINITY, z = 0.f;
+      for (int j = 0; j < my_n; ++j) {
+        ok = mbar_wait(my_sfull, (ph + (uint32_t)j) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        softmax_step<D>(t_s, t_o, j * kBN, limit, j == 0, scale_log2, m, z, my_pfull, bar_pfull_hi + 8 * x);
+      }
+      if (!ok) break;
+      // the next item's record (shown long ago) and this thread's row of it: the load travels under the epilogue
+      ok = wait_rec(k + 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      bool nrow_valid;
+      const int nc = row_rank(k + 1, nrow_valid);
+      if (my_n > 0) {
+        ok = mbar_wait(bar_ofinal + 8 * x, (ph >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const bool none = row_empty || !(z > 0.f);
+        const float inv = none ? 0.f : 1.f / z;
+        const float lse = none ? -INFINITY : (m + log2f(z)) * kLn2A;
+        const int4 b = rec_ld(k, 1);
+        const int hd = b.z;
+        const long long orow = (long long)b.w + x * tile_targets + t_local;
+        uint16_t* optr = out + (orow * H + hd * G + j_head) * D;
+#pragma unroll
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t o[32];
+          tmem_ld32(t_o + cc * 32, o);
+          tmem_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[i + 2 * e]) * inv, __uint_as_float(o[i + 2 * e + 1]) * inv);
+                w[e] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(optr + cc * 32 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        if (row_valid && lse_out) lse_out[(long long)(hd * G + j_head) * n_target_rows + orow] = lse;
+        tc_fence_before();
+        mbar_arrive(bar_odrained + 8 * x);
+        ph ^= 2u;
+      }
+      mbar_arrive(bar_itemfree + 8 * (k & 1u));                     // this thread is through with item k's record
+      ph = ((ph + (uint32_t)my_n) & 1u) | (ph & 2u) | ((k + 1) << 2);
+      c = nc; row_valid = nrow_valid;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) report(st, RELAXKV_ERR_TIMEOUT, KID_ATTN_SM100, (int)blockIdx.x, -2);
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 9) { tc_fence_after(); tmem_dealloc(tmem_base, kTmemCols); }
 }
 
 // Explicit lists (the paper's controlled configurations): per target the index of the last context entry
@@ -653,6 +1153,28 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D>::kDynamic) != cudaSuccess)
       return RELAXKV_ERR_CUDA;
     attr_done[dev].store(1, std::memory_order_release);
+  }
+  // Persistent form: where a block's work is short the turn-over between blocks is what there is to save (measured
+  // 3 % at an 8K context; nothing at 32K, where the chip runs at its power cap either way).
+  const relaxkv_tuning* tun = shape->h_tuning;
+  const int want_persist = tun ? tun->attention_persistent : 0;
+  if (n_splits == 1 && !plan.dense_ctx && (want_persist == 1 || (want_persist == 0 && max_tiles <= kPersistMaxTiles && grid > sms))) {
+    auto pk = attention_persist_kernel<D>;
+    static std::atomic<int> pattr_done[kMaxDevices];
+    if (!pattr_done[dev].load(std::memory_order_acquire)) {
+      if (cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, PersistSmem<D>::kDynamic) != cudaSuccess)
+        return RELAXKV_ERR_CUDA;
+      pattr_done[dev].store(1, std::memory_order_release);
+    }
+    int* counter = reinterpret_cast<int*>(plan.split_lse);          // unused by a one-split call: the work counter
+    if (cudaMemsetAsync(counter, 0, sizeof(int), stream) != cudaSuccess) return RELAXKV_ERR_CUDA;
+    long long pgrid = std::min<long long>(grid, sms);
+    if (tun && tun->attention_grid_blocks > 0) pgrid = std::min<long long>(grid, tun->attention_grid_blocks);
+    RELAXKV_RANGE("attention_persist_kernel");
+    pk<<<(unsigned)pgrid, kAttnThreads, PersistSmem<D>::kDynamic, stream>>>(
+        tm_q, tm_k, tm_v, plan.rt, mode, allow_empty, head_inner, H, Hkv, tile_targets, shape->softmax_scale * kLog2eA,
+        u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, (int)grid, counter, st);
+    return launch_ok();
   }
   RELAXKV_RANGE("attention_sm100_kernel");
   kern<<<dim3((unsigned)grid, (unsigned)n_splits), kAttnThreads, AttnSmem<D>::kDynamic, stream>>>(

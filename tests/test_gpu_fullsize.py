@@ -75,6 +75,32 @@ def test_qwen14b_32k_full_context_two_layers(ratio):
     run_full(inputs.qwen14b_32k("calibrated", ratio, n_layers=2), tile_targets=25, n_spread=24 if ratio == 0.15 else 12)
 
 
+def test_persistent_form_at_32k_equals_the_one_shot_kernel():
+    """A 32K layer (3 600 query-tile pairs x heads) through the persistent form, one block per SM as in production:
+    bit-identical to the one-shot kernel's output, and sampled rows against the oracle."""
+    from paper_2609_33503_b200 import binding as B
+    w = inputs.qwen14b_32k("calibrated", 0.15, n_layers=1)
+    case = Case(w)
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    f = case.fresh[0]
+    outs = []
+    for persistent in (2, 1):
+        s.shape.set_tuning(attention_persistent=persistent)
+        out = torch.zeros_like(f.q_new)
+        lse = torch.zeros(w.n_q_heads, f.q_new.shape[0], dtype=torch.float32, device=out.device)
+        s.attention(0, case.cache_views()[0], f.q_new, f.k_new, f.v_new, out, case.max_targets(0), case.max_ctx(), lse_out=lse)
+        st, detail = B.relaxkv_read_device_status()
+        assert st == 0, (st, detail)
+        outs.append((out, lse))
+    s.shape.set_tuning()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    rows = sampled_rows(f.q_new.shape[0], 50, 16, seed=3)
+    ref, _ = case.oracle_attention(0, 0, full_prefix=False, rows=rows)
+    mx, mean = attention_errors(outs[1][0][torch.from_numpy(rows.astype(np.int64)).to(out.device)], ref)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+
+
 def test_maximum_batch_of_64_requests():
     """The request table's limit (64 requests in one call) with ragged lengths from 1 token upwards:
     scores, anchors, sets, attention of every row, and the cache update against the oracle."""

@@ -269,6 +269,34 @@ def test_context_split_matches_oracle(case, n_splits):
         s.shape.set_tuning()
 
 
+@pytest.mark.parametrize("blocks", [1, 3, 0], ids=["one_block", "three_blocks", "one_per_sm"])
+def test_persistent_form_matches_oracle_and_the_one_shot_kernel(case, blocks):
+    """The persistent form of the attention kernel (one block walks many query-tile pairs, claimed from a counter):
+    forced on, with a single block walking every item, with three, and with one per SM; both context modes against
+    the oracle, bit-identical to the one-shot kernel, rows past a loosely bounded call's true count untouched."""
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    try:
+        for l in range(case.w.n_layers):
+            for full_prefix in (False, True):
+                mode = B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION
+                s.shape.set_tuning(attention_ctx_splits=1, attention_persistent=2)
+                ref, ref_lse = run_attention(case, s, l, mode, simt=False)
+                s.shape.set_tuning(attention_ctx_splits=1, attention_persistent=1, attention_grid_blocks=blocks)
+                out, lse = run_attention(case, s, l, mode, simt=False)
+                check_attention(case, l, out, lse, full_prefix)
+                assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
+        f = case.fresh[0]
+        n = f.q_new.shape[0]
+        q_pad = torch.cat([f.q_new, torch.zeros(7, *f.q_new.shape[1:], dtype=f.q_new.dtype, device=f.q_new.device)])
+        out = torch.full_like(q_pad, 3.0)
+        s.attention(0, case.cache_views()[0], q_pad, f.k_new, f.v_new, out, list(case.w.ctx_lens), list(case.w.ctx_lens))
+        assert_status_ok()
+        assert torch.all(out[n:] == 3.0)
+    finally:
+        s.shape.set_tuning()
+
+
 def test_attention_orders_agree_and_is_deterministic(case):
     """Update-then-attend from the cache equals mix-then-attend (Algorithm 1's order), bit for bit;
     two runs give identical bits."""
