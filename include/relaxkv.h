@@ -34,6 +34,10 @@
  *             the tensor-core kernels of later calls on that device return at once without writing their
  *             outputs, until the status word has been read (and thereby cleared): a caller that sees garbage
  *             should read the status word first.
+ * Graphs.     Every call only enqueues kernels, memsets and copies on `stream`, so calls can be recorded into a CUDA
+ *             graph; make the first call of each kind on a device outside the capture (it looks up device
+ *             addresses and opts kernels into large shared memory).  The host bounds and the choice of kernel form
+ *             are frozen into the graph.
  * Threads.    Calls may be made from several host threads; the per-device values the library looks up once
  *             (device addresses, attribute opt-ins) are published with atomics.  The status word is per device,
  *             not per thread or stream.

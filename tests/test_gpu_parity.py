@@ -297,6 +297,37 @@ def test_persistent_form_matches_oracle_and_the_one_shot_kernel(case, blocks):
         s.shape.set_tuning()
 
 
+@pytest.mark.parametrize("persistent", [2, 1], ids=["one_shot", "persistent"])
+def test_attention_call_replays_from_a_cuda_graph(persistent):
+    """Gather + attention captured into a CUDA graph (the persistent form also zeroes its work counter there) and
+    replayed twice give the bits of the eager call."""
+    case = Case(small_llama())
+    s = case.make_session()
+    s.build_active_sets(case.anchors_tensor())
+    s.shape.set_tuning(attention_ctx_splits=1, attention_persistent=persistent, attention_grid_blocks=2)
+    try:
+        eager, eager_lse = run_attention(case, s, 0, B().CTX_UNION, simt=False)
+        f = case.fresh[0]
+        out = torch.zeros_like(f.q_new)
+        lse = torch.zeros_like(eager_lse)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                s.attention(0, case.cache_views()[0], f.q_new, f.k_new, f.v_new, out, case.max_targets(0), case.max_ctx(),
+                            mode=B().CTX_UNION, lse_out=lse)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(2):
+            out.zero_(); lse.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert_status_ok()
+            assert torch.equal(out, eager) and torch.equal(lse, eager_lse)
+    finally:
+        s.shape.set_tuning()
+
+
 def test_attention_orders_agree_and_is_deterministic(case):
     """Update-then-attend from the cache equals mix-then-attend (Algorithm 1's order), bit for bit;
     two runs give identical bits."""
