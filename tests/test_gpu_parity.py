@@ -500,11 +500,14 @@ def test_list_attention_reduces_to_the_method(case):
     assert torch.equal(out, ref)
 
 
+@pytest.mark.parametrize("persistent", [0, 1], ids=["auto", "persistent"])
 @pytest.mark.parametrize("variant", ["global_targets", "layerwise_sparse", "global_sparse"])
-def test_controlled_configurations_match_oracle(case, variant):
+def test_controlled_configurations_match_oracle(case, variant, persistent):
     w = case.w
     rng = np.random.default_rng(5)
     s = case.make_session()
+    if persistent:                                # the persistent form of the kernel, two blocks walking all items
+        s.shape.set_tuning(attention_ctx_splits=1, attention_persistent=1, attention_grid_blocks=2)
     l = 0
     ctx_lists, tgt_lists = [], []
     for b in range(w.n_req):
