@@ -995,7 +995,7 @@ def run_ttft(args):
         phase[name] = phase.get(name, 0.0) + a.elapsed_time(b_) / args.steps
     total = t0.elapsed_time(t1) / args.steps
     ttft = total - phase["decode_step"]
-    weight_bytes = sum(v.numel() * 2 for wl in weights for k_, v in wl.items() if k_ != "w_gate_up") + w_head.numel() * 2
+    weight_bytes = sum(v.numel() * 2 for wl in weights for k_, v in wl.items() if k_ not in ("w_gate_up", "w_qkv")) + w_head.numel() * 2
     peaks = load_peaks()
     out = {"metric": "ttft_ms", "value": round(ttft, 3), "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": round(total, 3), "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",

@@ -347,11 +347,22 @@ relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, void* y, int64
                                float eps, relaxkv_stream stream);
 
 /* y = x weight^T (+ residual)      x [n_rows, n_in], weight [n_out, n_in] (the [out, in] layout),
- * residual NULL or [n_rows, n_out], y [n_rows, n_out] (may alias residual).  tcgen05 GEMM; calls of one to four
- * rows (a decode token, the row that goes through the output head) stream the weights once through a plain
- * HBM-bound kernel instead. */
+ * residual NULL or [n_rows, n_out], y [n_rows, n_out] (may alias residual).  tcgen05 GEMM: 256-row tiles on SM pairs
+ * for many rows; for 5 to 128 rows (the query's own tokens) 128 x 128 tiles whose K range is split over a
+ * thread-block cluster and summed through distributed shared memory in a fixed order, so that all SMs stream
+ * weights; calls of one to four rows (a decode token, the row that goes through the output head) stream the
+ * weights once through a plain HBM-bound kernel instead. */
 relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* residual, void* y,
                               int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream);
+
+/* The attention block's three input projections in one call: q = x Wq^T, k = x Wk^T, v = x Wv^T with
+ * w_qkv [n_q + 2 n_kv, n_in] = the rows of Wq, then Wk, then Wv (stacked once when the weights are loaded).
+ * x [n_rows, n_in]; q [n_rows, n_q], k and v [n_rows, n_kv]: three separate row-major buffers.  Same arithmetic per
+ * output element as relaxkv_linear.  Up to 128 rows (a decode token, the query's own tokens) this is ONE kernel that
+ * streams the stacked matrix once; for more rows it runs the three projections one after the other.
+ * n_q, n_kv, n_in multiples of 8. */
+relaxkv_status relaxkv_linear_qkv(const void* x, const void* w_qkv, void* q, void* k, void* v, int64_t n_rows,
+                                  int32_t n_q, int32_t n_kv, int32_t n_in, relaxkv_stream stream);
 
 /* out = silu(x Wg^T) * (x Wu^T) in one kernel (the MLP's first half): the gate and up projections and the
  * activation, with one rounding to bf16.  weight_tiled [2 * n_inter, n_in] holds, for every block t of 128

@@ -25,7 +25,7 @@ ENTRY_POINTS = (
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
     "relaxkv_list_attention", "relaxkv_cache_attention",
-    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_swiglu", "relaxkv_rope",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_qkv", "relaxkv_linear_swiglu", "relaxkv_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
 
@@ -319,6 +319,22 @@ def relaxkv_linear(x: torch.Tensor, weight: torch.Tensor, y: torch.Tensor, resid
     """y = x weight^T (+ residual); weight is [n_out, n_in]."""
     _check(lib().relaxkv_linear(_ptr(x), _ptr(weight), _ptr(residual), _ptr(y), ctypes.c_int64(x.shape[0]),
                                 int(weight.shape[0]), int(weight.shape[1]), _stream(stream)), "relaxkv_linear")
+
+
+def stack_qkv(wq: torch.Tensor, wk: torch.Tensor, wv: torch.Tensor) -> torch.Tensor:
+    """[Wq; Wk; Wv] along the output features: the weight layout relaxkv_linear_qkv reads (a copy, made once when the
+    weights are loaded)."""
+    return torch.cat([wq, wk, wv], dim=0).contiguous()
+
+
+def relaxkv_linear_qkv(x: torch.Tensor, w_qkv: torch.Tensor, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, stream=None) -> None:
+    """q, k, v = x Wq^T, x Wk^T, x Wv^T with w_qkv = [Wq; Wk; Wv] stacked along the output features.
+    q [n, n_q] (or any contiguous view of it), k and v [n, n_kv]."""
+    n = x.shape[0]
+    n_q, n_kv = q.numel() // max(n, 1), k.numel() // max(n, 1)
+    assert w_qkv.shape[0] == n_q + 2 * n_kv and v.numel() == k.numel()
+    _check(lib().relaxkv_linear_qkv(_ptr(x), _ptr(w_qkv), _ptr(q), _ptr(k), _ptr(v), ctypes.c_int64(n), int(n_q), int(n_kv),
+                                    int(w_qkv.shape[1]), _stream(stream)), "relaxkv_linear_qkv")
 
 
 def tile_gate_up(w_gate_up: torch.Tensor) -> torch.Tensor:

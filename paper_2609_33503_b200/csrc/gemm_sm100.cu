@@ -6,6 +6,7 @@
 // lane) drain tile i while the tensor pipe works on tile i+1.  Tiles are walked in groups of 16 row tiles so
 // that a wave's working set (x rows + W rows) stays in L2.
 #include "common.cuh"
+#include "gemm_skinny.cuh"
 #include "gemv.cuh"
 #include "sm100_ptx.cuh"
 #include <algorithm>
@@ -407,6 +408,17 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
   if (n_rows == 0) return RELAXKV_OK;
   if (n_rows <= kGemvMaxRows)       // a decode token: stream the weights once, no 128-row tiles
     return launch_gemv(x, weight, residual, y, (int)n_rows, n_out, n_in, swiglu, static_cast<cudaStream_t>(stream_));
+  if (n_rows <= kSkinnyMaxRows && !swiglu && skinny_tiles(n_out) <= sm_count_of_current_device()) {
+    // one row tile and no more column tiles than SMs (the query's tokens through a 5120-wide projection): 128 x 128
+    // tiles, K split over a cluster so that about all SMs stream weights.  (The fused gate/up projection has 272 such
+    // tiles at the model shapes and keeps the large kernel.)
+    SkinnyOut outs = {};
+    outs.y[0] = static_cast<uint16_t*>(y);
+    outs.residual[0] = static_cast<const uint16_t*>(residual);
+    outs.col0[0] = 0; outs.col0[1] = n_out;
+    outs.n = 1;
+    return launch_gemm_skinny(x, weight, outs, (int)n_rows, n_out, n_in, static_cast<cudaStream_t>(stream_));
+  }
   // SM pairs (256-row tiles) unless that would leave a large share of the last tile row empty: with an odd number of
   // 128-row tiles, seven at most, the second block of the last pair would compute padding only (>= 1/8 of the work),
   // and the single-block kernel (128 x 256 tiles) is used.
@@ -469,6 +481,37 @@ extern "C" relaxkv_status relaxkv_linear(const void* x, const void* weight, cons
                                          int64_t n_rows, int32_t n_out, int32_t n_in, relaxkv_stream stream_) {
   RELAXKV_RANGE("relaxkv_linear");
   return launch_gemm(x, weight, residual, y, n_rows, n_out, n_in, 0, stream_);
+}
+
+extern "C" relaxkv_status relaxkv_linear_qkv(const void* x, const void* w_qkv, void* q, void* k, void* v, int64_t n_rows,
+                                             int32_t n_q, int32_t n_kv, int32_t n_in, relaxkv_stream stream_) {
+  RELAXKV_RANGE("relaxkv_linear_qkv");
+  if (!x || !w_qkv || !q || !k || !v || !aligned16(x) || !aligned16(w_qkv) || !aligned16(q) || !aligned16(k) || !aligned16(v))
+    return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_q < 8 || n_kv < 8 || n_in < 8 || (n_q % 8) || (n_kv % 8) || (n_in % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  const int n_out = n_q + 2 * n_kv;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (n_rows <= kGemvMaxRows) {
+    GemvOut outs = {};
+    outs.y[0] = static_cast<uint16_t*>(q); outs.y[1] = static_cast<uint16_t*>(k); outs.y[2] = static_cast<uint16_t*>(v);
+    outs.col0[0] = 0; outs.col0[1] = n_q; outs.col0[2] = n_q + n_kv; outs.col0[3] = n_out;
+    outs.n = 3;
+    return launch_gemv_segments(x, w_qkv, outs, (int)n_rows, n_out, n_in, stream);
+  }
+  if (n_rows <= kSkinnyMaxRows && skinny_tiles(n_out) <= sm_count_of_current_device()) {
+    SkinnyOut outs = {};
+    outs.y[0] = static_cast<uint16_t*>(q); outs.y[1] = static_cast<uint16_t*>(k); outs.y[2] = static_cast<uint16_t*>(v);
+    outs.col0[0] = 0; outs.col0[1] = n_q; outs.col0[2] = n_q + n_kv; outs.col0[3] = n_out;
+    outs.n = 3;
+    return launch_gemm_skinny(x, w_qkv, outs, (int)n_rows, n_out, n_in, stream);
+  }
+  // many rows: the three projections one after the other (each is at the tensor peak on its own)
+  const uint16_t* w = static_cast<const uint16_t*>(w_qkv);
+  relaxkv_status rc = launch_gemm(x, w, nullptr, q, n_rows, n_q, n_in, 0, stream_);
+  if (rc == RELAXKV_OK) rc = launch_gemm(x, w + (size_t)n_q * n_in, nullptr, k, n_rows, n_kv, n_in, 0, stream_);
+  if (rc == RELAXKV_OK) rc = launch_gemm(x, w + (size_t)(n_q + n_kv) * n_in, nullptr, v, n_rows, n_kv, n_in, 0, stream_);
+  return rc;
 }
 
 extern "C" relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weight_tiled, void* y, int64_t n_rows,

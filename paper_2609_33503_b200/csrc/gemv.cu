@@ -23,10 +23,12 @@ __device__ __forceinline__ void unpack8_gemv(const uint4& v, float* f) {
 // SWIGLU = 0: y[m, n] = sum_k x[m, k] w[n, k] (+ residual[m, n])          w [n_out, K]
 // SWIGLU = 1: y[m, f] = silu(sum_k x w[g(f), k]) * (sum_k x w[g(f) + 128, k])   with g(f) = (f / 128) * 256 + f % 128
 //             (the gate rows of every block of 128 features are followed by its up rows); n_out counts the features f
-template <int M, int SWIGLU>
+// SEG = 1: the features are the rows of several stacked weight matrices (the fused Q/K/V projection) and segment i,
+//          features [col0[i], col0[i + 1]), is written to its own buffer outs.y[i] of that width; y is unused.
+template <int M, int SWIGLU, int SEG>
 __global__ void __launch_bounds__(kGemvThreads)
 gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, const uint16_t* __restrict__ residual,
-            uint16_t* __restrict__ y, int n_out, int K) {
+            uint16_t* __restrict__ y, int n_out, int K, const GemvOut outs) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int f0 = blockIdx.x * kGemvFeatPerBlock + warp * kGemvFeatPerWarp;
   constexpr int R = SWIGLU ? 2 * kGemvFeatPerWarp : kGemvFeatPerWarp;      // weight rows this warp streams
@@ -81,24 +83,28 @@ gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, cons
             }
           }
         }
-        const long long o = (long long)m * n_out + f;
-        if (!SWIGLU && residual) v += bf16_bits_to_float(residual[o]);
-        const __nv_bfloat16 h = __float2bfloat16(v);
-        y[o] = *reinterpret_cast<const uint16_t*>(&h);
+        const __nv_bfloat16 h = __float2bfloat16((!SWIGLU && !SEG && residual) ? v + bf16_bits_to_float(residual[(long long)m * n_out + f]) : v);
+        if (SEG) {
+          int sg = 0;
+          while (sg + 1 < outs.n && f >= outs.col0[sg + 1]) ++sg;
+          outs.y[sg][(long long)m * (outs.col0[sg + 1] - outs.col0[sg]) + (f - outs.col0[sg])] = *reinterpret_cast<const uint16_t*>(&h);
+        } else {
+          y[(long long)m * n_out + f] = *reinterpret_cast<const uint16_t*>(&h);
+        }
       }
     }
   }
 }
 
-template <int SWIGLU>
+template <int SWIGLU, int SEG>
 static relaxkv_status launch_m(const uint16_t* x, const uint16_t* w, const uint16_t* residual, uint16_t* y, int n_rows,
-                               int n_out, int K, cudaStream_t stream) {
+                               int n_out, int K, const GemvOut& outs, cudaStream_t stream) {
   const unsigned blocks = (unsigned)((n_out + kGemvFeatPerBlock - 1) / kGemvFeatPerBlock);
   switch (n_rows) {
-    case 1: gemv_kernel<1, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
-    case 2: gemv_kernel<2, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
-    case 3: gemv_kernel<3, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
-    case 4: gemv_kernel<4, SWIGLU><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K); break;
+    case 1: gemv_kernel<1, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 2: gemv_kernel<2, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 3: gemv_kernel<3, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 4: gemv_kernel<4, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
     default: return RELAXKV_ERR_INVALID_ARG;
   }
   return launch_ok();
@@ -107,11 +113,19 @@ static relaxkv_status launch_m(const uint16_t* x, const uint16_t* w, const uint1
 relaxkv_status launch_gemv(const void* x, const void* weight, const void* residual, void* y, int n_rows, int n_out,
                            int n_in, int swiglu, cudaStream_t stream) {
   RELAXKV_RANGE("gemv_kernel");
+  const GemvOut none = {};
   if (swiglu)
-    return launch_m<1>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), nullptr,
-                       static_cast<uint16_t*>(y), n_rows, n_out / 2, n_in, stream);
-  return launch_m<0>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight),
-                     static_cast<const uint16_t*>(residual), static_cast<uint16_t*>(y), n_rows, n_out, n_in, stream);
+    return launch_m<1, 0>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), nullptr,
+                          static_cast<uint16_t*>(y), n_rows, n_out / 2, n_in, none, stream);
+  return launch_m<0, 0>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight),
+                        static_cast<const uint16_t*>(residual), static_cast<uint16_t*>(y), n_rows, n_out, n_in, none, stream);
+}
+
+relaxkv_status launch_gemv_segments(const void* x, const void* weight, const GemvOut& outs, int n_rows, int n_out, int n_in,
+                                    cudaStream_t stream) {
+  RELAXKV_RANGE("gemv_kernel");
+  return launch_m<0, 1>(static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), nullptr, nullptr, n_rows, n_out,
+                        n_in, outs, stream);
 }
 
 }  // namespace relaxkv

@@ -75,8 +75,9 @@ class QueryPass:
     def _block(self, l, w, cache, h, x, a, q, k, v, o, gu, m, h_out, pos, cu, counts, shape, attend, rec):
         blk, D, n = self.blk, self.D, h.shape[0]
         rec("norm", lambda: B.relaxkv_rmsnorm(h, w["w_in_norm"], x, blk.eps))
-        rec("qkv_proj", lambda: (B.relaxkv_linear(x, w["wq"], q.view(n, -1)), B.relaxkv_linear(x, w["wk"], k.view(n, -1)),
-                                 B.relaxkv_linear(x, w["wv"], v.view(n, -1))))
+        if "w_qkv" not in w:                            # weight-loading step, once per layer: [Wq; Wk; Wv] stacked
+            w["w_qkv"] = B.stack_qkv(w["wq"], w["wk"], w["wv"])
+        rec("qkv_proj", lambda: B.relaxkv_linear_qkv(x, w["w_qkv"], q.view(n, -1), k.view(n, -1), v.view(n, -1)))
         if "w_q_norm" in w:
             rec("norm", lambda: (B.relaxkv_rmsnorm(q.view(-1, D), w["w_q_norm"], q.view(-1, D), blk.eps),
                                  B.relaxkv_rmsnorm(k.view(-1, D), w["w_k_norm"], k.view(-1, D), blk.eps)))

@@ -54,6 +54,30 @@ def _check_linear(M, N, K, res):
     torch.testing.assert_close(y.float(), (x.float() @ w.float().T + (r.float() if res else 0)), rtol=2e-2, atol=2e-2)
 
 
+@pytest.mark.parametrize("M", [1, 3, 5, 64, 128, 300])
+@pytest.mark.parametrize("n_q,n_kv,K", [(512, 128, 512), (5120, 1024, 5120), (320, 72, 264)])
+def test_linear_qkv_writes_the_three_projections(M, n_q, n_kv, K):
+    """The fused Q/K/V projection (stacked weight, three output buffers) through its three routes - the streaming
+    kernel (1-4 rows), the cluster split-K kernel (5-128 rows: segment boundaries inside a tile at the odd shape), three
+    large GEMMs (300 rows) - against the oracle's linear per projection; bytes around the outputs stay untouched."""
+    x = rnd(M, K, seed=11)
+    wq, wk, wv = rnd(n_q, K, scale=K ** -0.5, seed=12), rnd(n_kv, K, scale=K ** -0.5, seed=13), rnd(n_kv, K, scale=K ** -0.5, seed=14)
+    w_qkv = B().stack_qkv(wq, wk, wv)
+    bufs = [torch.full((M + 2, n), 7.0, dtype=torch.bfloat16, device="cuda") for n in (n_q, n_kv, n_kv)]
+    q, k, v = (b[1:M + 1] for b in bufs)
+    B().relaxkv_linear_qkv(x, w_qkv, q, k, v)
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+    for out, w, buf in ((q, wq, bufs[0]), (k, wk, bufs[1]), (v, wv, bufs[2])):
+        ref = blk.linear(blk.f64(bits(x)), blk.f64(bits(w)), None)
+        close(out, ref, abs_floor=2e-3)
+        assert torch.all(buf[0] == 7.0) and torch.all(buf[M + 1] == 7.0)
+        if M <= 4:                                   # the streaming kernel: same arithmetic as the single projection
+            one = torch.empty_like(out)
+            B().relaxkv_linear(x, w, one)
+            assert torch.equal(one, out)
+
+
 def test_linear_at_the_benchmark_shapes():
     """The projections at the sizes the repair loop runs them for the 32K Qwen3-14B-shaped stack: 18 000 active rows
     through a 5120 -> 5120 projection with residual (SM pairs) and the fused gate/up projection of 5120 -> 2 x 17408 on
