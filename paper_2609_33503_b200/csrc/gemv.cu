@@ -25,12 +25,17 @@ __device__ __forceinline__ void unpack8_gemv(const uint4& v, float* f) {
 //             (the gate rows of every block of 128 features are followed by its up rows); n_out counts the features f
 // SEG = 1: the features are the rows of several stacked weight matrices (the fused Q/K/V projection) and segment i,
 //          features [col0[i], col0[i + 1]), is written to its own buffer outs.y[i] of that width; y is unused.
-template <int M, int SWIGLU, int SEG>
+// KS > 1: KS warps share a warp's features and split K among them (partial sums added through shared memory in a
+//         fixed order): a matrix of a few tens of MB then has four times as many, four times shorter dependent load
+//         chains, which is what bounds such a launch (not bandwidth).
+template <int M, int SWIGLU, int SEG, int KS>
 __global__ void __launch_bounds__(kGemvThreads)
 gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, const uint16_t* __restrict__ residual,
             uint16_t* __restrict__ y, int n_out, int K, const GemvOut outs) {
+  constexpr int kWarps = kGemvThreads / 32, kGroups = kWarps / KS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int f0 = blockIdx.x * kGemvFeatPerBlock + warp * kGemvFeatPerWarp;
+  const int grp = warp / KS, kp = warp % KS;
+  const int f0 = (blockIdx.x * kGroups + grp) * kGemvFeatPerWarp;
   constexpr int R = SWIGLU ? 2 * kGemvFeatPerWarp : kGemvFeatPerWarp;      // weight rows this warp streams
   const uint16_t* wr[R];
 #pragma unroll
@@ -44,8 +49,10 @@ gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, cons
   for (int r = 0; r < R; ++r)
 #pragma unroll
     for (int m = 0; m < M; ++m) acc[r][m] = 0.f;
+  const int k_part = (KS == 1) ? K : ((K + KS * 256 - 1) / (KS * 256)) * 256;      // this warp's share of K
+  const int k_lo = kp * k_part, k_hi = min(K, k_lo + k_part);
 #pragma unroll 4
-  for (int k = lane * 8; k < K; k += 32 * 8) {
+  for (int k = k_lo + lane * 8; k < k_hi; k += 32 * 8) {
     uint4 wv[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) wv[r] = __ldg(reinterpret_cast<const uint4*>(wr[r] + k));     // all loads first
@@ -66,6 +73,26 @@ gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, cons
   for (int r = 0; r < R; ++r)
 #pragma unroll
     for (int m = 0; m < M; ++m) acc[r][m] = warp_reduce_sum(acc[r][m]);
+  if (KS > 1) {
+    __shared__ float part[kWarps][R][M];
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int m = 0; m < M; ++m) part[warp][r][m] = acc[r][m];
+    }
+    __syncthreads();
+    if (kp != 0) return;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        float v = 0.f;
+#pragma unroll
+        for (int q = 0; q < KS; ++q) v += part[grp * KS + q][r][m];          // fixed order
+        acc[r][m] = v;
+      }
+  }
   if (lane < kGemvFeatPerWarp) {
     const int f = f0 + lane;
     if (f < n_out) {
@@ -96,18 +123,30 @@ gemv_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, cons
   }
 }
 
-template <int SWIGLU, int SEG>
-static relaxkv_status launch_m(const uint16_t* x, const uint16_t* w, const uint16_t* residual, uint16_t* y, int n_rows,
-                               int n_out, int K, const GemvOut& outs, cudaStream_t stream) {
-  const unsigned blocks = (unsigned)((n_out + kGemvFeatPerBlock - 1) / kGemvFeatPerBlock);
+constexpr long long kGemvSplitKBelowBytes = 256ll << 20;     // matrices below this size split K over four warps
+
+template <int SWIGLU, int SEG, int KS>
+static relaxkv_status launch_mk(const uint16_t* x, const uint16_t* w, const uint16_t* residual, uint16_t* y, int n_rows,
+                                int n_out, int K, const GemvOut& outs, cudaStream_t stream) {
+  constexpr int feat_per_block = kGemvFeatPerBlock / KS;
+  const unsigned blocks = (unsigned)((n_out + feat_per_block - 1) / feat_per_block);
   switch (n_rows) {
-    case 1: gemv_kernel<1, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
-    case 2: gemv_kernel<2, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
-    case 3: gemv_kernel<3, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
-    case 4: gemv_kernel<4, SWIGLU, SEG><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 1: gemv_kernel<1, SWIGLU, SEG, KS><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 2: gemv_kernel<2, SWIGLU, SEG, KS><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 3: gemv_kernel<3, SWIGLU, SEG, KS><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
+    case 4: gemv_kernel<4, SWIGLU, SEG, KS><<<blocks, kGemvThreads, 0, stream>>>(x, w, residual, y, n_out, K, outs); break;
     default: return RELAXKV_ERR_INVALID_ARG;
   }
   return launch_ok();
+}
+
+template <int SWIGLU, int SEG>
+static relaxkv_status launch_m(const uint16_t* x, const uint16_t* w, const uint16_t* residual, uint16_t* y, int n_rows,
+                               int n_out, int K, const GemvOut& outs, cudaStream_t stream) {
+  const long long bytes = (long long)(SWIGLU ? 2 : 1) * n_out * K * 2;
+  if (bytes < kGemvSplitKBelowBytes && K >= 4 * 256)
+    return launch_mk<SWIGLU, SEG, 4>(x, w, residual, y, n_rows, n_out, K, outs, stream);
+  return launch_mk<SWIGLU, SEG, 1>(x, w, residual, y, n_rows, n_out, K, outs, stream);
 }
 
 relaxkv_status launch_gemv(const void* x, const void* weight, const void* residual, void* y, int n_rows, int n_out,
