@@ -382,6 +382,15 @@ relaxkv_status relaxkv_linear_swiglu(const void* x, const void* weight_tiled, vo
 relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
                             float theta, relaxkv_stream stream);
 
+/* The per-head RMSNorm of the projected queries and keys (models that have one; pass NULL weights otherwise) followed by
+ * the rotary embedding, on q [n_rows, n_q_heads, head_dim] and k [n_rows, n_kv_heads, head_dim] in place, in ONE
+ * launch: the same results as relaxkv_rmsnorm on the head vectors of q and of k followed by relaxkv_rope on q and on
+ * k (the normalised values are rounded to bf16 in between, as a store would), meant for the few rows of a query pass
+ * or a decode step, where four launches cost more than their work.  w_q_norm, w_k_norm: [head_dim] or both NULL. */
+relaxkv_status relaxkv_qk_norm_rope(void* q, void* k, int64_t n_rows, int32_t n_q_heads, int32_t n_kv_heads,
+                                    int32_t head_dim, const void* w_q_norm, const void* w_k_norm, float eps,
+                                    const int32_t* positions, float theta, relaxkv_stream stream);
+
 /* out[r, i] = silu(gate_up[r, i]) * gate_up[r, n_inter + i]      gate_up [n_rows, 2*n_inter], out [n_rows, n_inter] */
 relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t n_rows, int32_t n_inter, relaxkv_stream stream);
 

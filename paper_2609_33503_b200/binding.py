@@ -25,7 +25,7 @@ ENTRY_POINTS = (
     "relaxkv_sparse_ctx_attention_simt", "relaxkv_read_device_status", "relaxkv_select_topk",
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
     "relaxkv_list_attention", "relaxkv_cache_attention",
-    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_qkv", "relaxkv_linear_swiglu", "relaxkv_rope",
+    "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_qkv", "relaxkv_linear_swiglu", "relaxkv_rope", "relaxkv_qk_norm_rope",
     "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
 )
 
@@ -358,6 +358,15 @@ def relaxkv_rope(x: torch.Tensor, positions: torch.Tensor, theta: float, stream=
     """In place on x [rows, heads, D]; positions int32 [rows]."""
     _check(lib().relaxkv_rope(_ptr(x), ctypes.c_int64(x.shape[0]), int(x.shape[1]), int(x.shape[2]), _ptr(positions),
                               ctypes.c_float(theta), _stream(stream)), "relaxkv_rope")
+
+
+def relaxkv_qk_norm_rope(q: torch.Tensor, k: torch.Tensor, positions: torch.Tensor, theta: float,
+                         w_q_norm: Optional[torch.Tensor] = None, w_k_norm: Optional[torch.Tensor] = None, eps: float = 1e-6,
+                         stream=None) -> None:
+    """Per-head RMSNorm (when weights are given) and rotary embedding of q [n, H, D] and k [n, H_kv, D], in place."""
+    _check(lib().relaxkv_qk_norm_rope(_ptr(q), _ptr(k), ctypes.c_int64(q.shape[0]), int(q.shape[1]), int(k.shape[1]),
+                                      int(q.shape[2]), _ptr(w_q_norm), _ptr(w_k_norm), ctypes.c_float(eps), _ptr(positions),
+                                      ctypes.c_float(theta), _stream(stream)), "relaxkv_qk_norm_rope")
 
 
 def relaxkv_swiglu(gate_up: torch.Tensor, out: torch.Tensor, stream=None) -> None:

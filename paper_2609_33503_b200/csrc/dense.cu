@@ -111,6 +111,55 @@ __global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads,
   }
 }
 
+// Per-head RMSNorm (optional) and rotary embedding of the projected queries and keys of a few rows in ONE launch
+// (the query's own tokens, a decode token: four launches of a few microseconds otherwise).  One block per row: the
+// first D/2 threads compute the row's (cos, sin) table once, then every warp takes heads (query heads first, then KV
+// heads); a lane holds D/32 consecutive dims, its rotation partner sits 16 lanes away.  Between the two steps the
+// values are rounded to bf16, as they would be if the normalised heads had been stored and read back.
+template <int D>
+__global__ void __launch_bounds__(128)
+head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq, int Hkv, const uint16_t* __restrict__ wq,
+                      const uint16_t* __restrict__ wk, float eps, const int* __restrict__ positions, float log2_theta) {
+  constexpr int DPL = D / 32, half = D / 2;
+  __shared__ float cs_s[half], sn_s[half];
+  const long long row = blockIdx.x;
+  if (threadIdx.x < half) {
+    const int i = threadIdx.x;
+    const double inv_freq = exp2(-(double)log2_theta * (2.0 * i / D));
+    double ang = (double)positions[row] * inv_freq;
+    ang -= 6.283185307179586 * floor(ang * 0.15915494309189535);
+    sincosf((float)ang, &sn_s[i], &cs_s[i]);
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int d0 = lane * DPL;                                  // this lane's dims d0 .. d0 + DPL - 1
+  const bool low = d0 < half;                                 // first half of the head vector: partner is + D/2
+  for (int h = warp; h < Hq + Hkv; h += 4) {
+    uint16_t* v = (h < Hq) ? q + (row * Hq + h) * D : k + (row * Hkv + (h - Hq)) * D;
+    const uint16_t* w = (h < Hq) ? wq : wk;
+    float f[DPL];
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) f[e] = bf16_bits_to_float(v[d0 + e]);
+    if (w != nullptr) {
+      float ss = 0.f;
+#pragma unroll
+      for (int e = 0; e < DPL; ++e) ss = fmaf(f[e], f[e], ss);
+      ss = warp_reduce_sum(ss);
+      const float inv = rsqrtf(ss / (float)D + eps);
+#pragma unroll
+      for (int e = 0; e < DPL; ++e) f[e] = __bfloat162float(__float2bfloat16(f[e] * inv * bf16_bits_to_float(w[d0 + e])));
+    }
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) {
+      const float other = __shfl_xor_sync(0xffffffffu, f[e], 16);        // dim d0 + e -/+ D/2
+      const int i = (d0 + e) % half;
+      const float r = low ? f[e] * cs_s[i] - other * sn_s[i] : f[e] * cs_s[i] + other * sn_s[i];
+      const __nv_bfloat16 hb = __float2bfloat16(r);
+      v[d0 + e] = *reinterpret_cast<const uint16_t*>(&hb);
+    }
+  }
+}
+
 // out[r, i] = silu(gu[r, i]) * gu[r, I + i]
 __global__ void swiglu_kernel(const uint16_t* __restrict__ gu, uint16_t* __restrict__ out, long long rows, int I) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -204,6 +253,25 @@ extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads,
   const long long n = n_rows * (head_dim / 16);
   rope_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<uint16_t*>(x), n_rows, n_heads, head_dim, positions, log2f(theta));
+  return launch_ok();
+}
+
+extern "C" relaxkv_status relaxkv_qk_norm_rope(void* q, void* k, int64_t n_rows, int32_t n_q_heads, int32_t n_kv_heads,
+                                               int32_t head_dim, const void* w_q_norm, const void* w_k_norm, float eps,
+                                               const int32_t* positions, float theta, relaxkv_stream stream) {
+  RELAXKV_RANGE("relaxkv_qk_norm_rope");
+  if (!q || !k || !positions || !aligned16(q) || !aligned16(k) || !(theta > 1.f) || !(eps >= 0.f)) return RELAXKV_ERR_INVALID_ARG;
+  if ((w_q_norm == nullptr) != (w_k_norm == nullptr)) return RELAXKV_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_q_heads < 1 || n_kv_heads < 1 || (head_dim != 64 && head_dim != 128)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  if (n_rows == 0) return RELAXKV_OK;
+  if (n_rows > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128)
+    head_norm_rope_kernel<128><<<(unsigned)n_rows, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads,
+        static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
+  else
+    head_norm_rope_kernel<64><<<(unsigned)n_rows, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads,
+        static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
   return launch_ok();
 }
 

@@ -4,8 +4,8 @@ cache, one attention per layer; reproducibility appendix: query prefill and the 
 region).  Call sequencing over torch buffers only; every operation runs in the CUDA kernels behind
 `binding`.
 
-Per layer the query's rows run the decoder block: RMSNorm, Q/K/V projections, per-head Q/K norm where the model has
-one, rotary embedding at positions T_c, T_c + 1, ..., their K/V are appended to the cache behind the context rows,
+Per layer the query's rows run the decoder block: RMSNorm, the stacked Q/K/V projection, per-head Q/K norm where the
+model has one and rotary embedding at positions T_c, T_c + 1, ... (one launch), their K/V are appended to the cache behind the context rows,
 then causal attention over [context, query] (`relaxkv_query_prefill_attention`, which can emit the context scores of
 that very pass), output projection + residual, MLP + residual.  The decode step is the same block for one new token
 (the projections take the streaming one-row kernel), followed by the final norm and the output head.
@@ -78,10 +78,7 @@ class QueryPass:
         if "w_qkv" not in w:                            # weight-loading step, once per layer: [Wq; Wk; Wv] stacked
             w["w_qkv"] = B.stack_qkv(w["wq"], w["wk"], w["wv"])
         rec("qkv_proj", lambda: B.relaxkv_linear_qkv(x, w["w_qkv"], q.view(n, -1), k.view(n, -1), v.view(n, -1)))
-        if "w_q_norm" in w:
-            rec("norm", lambda: (B.relaxkv_rmsnorm(q.view(-1, D), w["w_q_norm"], q.view(-1, D), blk.eps),
-                                 B.relaxkv_rmsnorm(k.view(-1, D), w["w_k_norm"], k.view(-1, D), blk.eps)))
-        rec("rope", lambda: (B.relaxkv_rope(q, pos, blk.rope_theta), B.relaxkv_rope(k, pos, blk.rope_theta)))
+        rec("rope", lambda: B.relaxkv_qk_norm_rope(q, k, pos, blk.rope_theta, w.get("w_q_norm"), w.get("w_k_norm"), blk.eps))
         rec("append_kv", lambda: B.relaxkv_scatter_kv_lists(shape, cache, k, v, pos, cu, counts))
         rec("attention", attend)
         rec("o_proj", lambda: B.relaxkv_linear(o.view(n, -1), w["wo"], a, residual=h))

@@ -134,6 +134,33 @@ def test_rmsnorm_rope_swiglu():
     close(out, blk.swiglu(blk.f64(bits(gu))), abs_floor=1e-3)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("with_norm", [True, False])
+def test_qk_norm_rope_in_one_launch(D, with_norm):
+    """Per-head RMSNorm (optional) + rotary embedding of q and k in one launch against the oracle's rmsnorm -> bf16
+    storage -> rope per tensor, and against the library's own separate calls (equal up to the last bf16 bit of the
+    normalised values); neighbouring rows untouched."""
+    n, H, Hkv, theta, eps = 37, 5, 2, 1e6, 1e-6
+    qb, kb = rnd(n + 2, H, D, seed=31, scale=2.0), rnd(n + 2, Hkv, D, seed=32, scale=2.0)
+    q0, k0 = qb.clone(), kb.clone()
+    wq, wk = (rnd(D, seed=33), rnd(D, seed=34)) if with_norm else (None, None)
+    pos = torch.tensor(np.random.default_rng(1).integers(0, 70000, size=n).astype(np.int32)).cuda()
+    q, k = qb[1:n + 1], kb[1:n + 1]
+    B().relaxkv_qk_norm_rope(q, k, pos, theta, wq, wk, eps)
+    for got, x0, w, heads in ((q, q0[1:n + 1], wq, H), (k, k0[1:n + 1], wk, Hkv)):
+        x = blk.f64(bits(x0))
+        if with_norm:
+            x = bf16_round(blk.rmsnorm(x.reshape(n * heads, D), blk.f64(bits(w)), eps)).reshape(n, heads, D)
+        ref = blk.rope(x, pos.cpu().numpy(), theta)
+        close(got, ref, abs_floor=4e-3 if with_norm else 2e-3)
+        two = x0.clone()
+        if with_norm:
+            B().relaxkv_rmsnorm(two.view(-1, D), w, two.view(-1, D), eps)
+        B().relaxkv_rope(two, pos, theta)
+        assert float((two.float() - got.float()).abs().max()) <= 2.0 ** -6 * float(two.float().abs().max())
+    assert torch.equal(qb[0], q0[0]) and torch.equal(qb[n + 1], q0[n + 1]) and torch.equal(kb[0], k0[0]) and torch.equal(kb[n + 1], k0[n + 1])
+
+
 def test_target_positions_and_row_carry():
     from tests.harness import Case
     w = inputs.scaled_down(inputs.qwen14b_32k("calibrated"), (640, 900), (9, 17), n_layers=3, chunk=128)
