@@ -112,13 +112,16 @@ __global__ void rope_kernel(uint16_t* __restrict__ x, long long rows, int heads,
 }
 
 // Per-head RMSNorm (optional) and rotary embedding of the projected queries and keys of a few rows in ONE launch
-// (the query's own tokens, a decode token: four launches of a few microseconds otherwise).  One block per row: the
-// first D/2 threads compute the row's (cos, sin) table once, then every warp takes heads (query heads first, then KV
-// heads); a lane holds D/32 consecutive dims, its rotation partner sits 16 lanes away.  Between the two steps the
+// (the query's own tokens, a decode token: four launches of a few microseconds otherwise; for the repair loop's many
+// rows: one pass over q and k instead of two).  One block per (row, four heads): the first D/2 threads compute the
+// row's (cos, sin) table, then every warp takes one head (query heads first, then KV
+// heads); a lane holds D/32 consecutive dims, its rotation partner sits 16 lanes away.  Grid: (rows, groups of heads):
+// four heads per block for a few rows (all warps busy at once), all heads in one block for many rows (the table's
+// double-precision arithmetic, about 3 k clk per block, is then paid once per row).  Between the two steps the
 // values are rounded to bf16, as they would be if the normalised heads had been stored and read back.
 template <int D>
 __global__ void __launch_bounds__(128)
-head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq, int Hkv, const uint16_t* __restrict__ wq,
+head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq, int Hkv, int heads_per_block, const uint16_t* __restrict__ wq,
                       const uint16_t* __restrict__ wk, float eps, const int* __restrict__ positions, float log2_theta) {
   constexpr int DPL = D / 32, half = D / 2;
   __shared__ float cs_s[half], sn_s[half];
@@ -134,12 +137,20 @@ head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int d0 = lane * DPL;                                  // this lane's dims d0 .. d0 + DPL - 1
   const bool low = d0 < half;                                 // first half of the head vector: partner is + D/2
-  for (int h = warp; h < Hq + Hkv; h += 4) {
+  // heads of this block: [blockIdx.y * heads_per_block, + heads_per_block), one per warp and round
+  const int h_end = min(Hq + Hkv, ((int)blockIdx.y + 1) * heads_per_block);
+  for (int h = blockIdx.y * heads_per_block + warp; h < h_end; h += 4) {
     uint16_t* v = (h < Hq) ? q + (row * Hq + h) * D : k + (row * Hkv + (h - Hq)) * D;
     const uint16_t* w = (h < Hq) ? wq : wk;
     float f[DPL];
-#pragma unroll
-    for (int e = 0; e < DPL; ++e) f[e] = bf16_bits_to_float(v[d0 + e]);
+    if constexpr (DPL == 4) {                                  // one 8-byte access per lane
+      const uint2 raw = *reinterpret_cast<const uint2*>(v + d0);
+      f[0] = __uint_as_float(raw.x << 16); f[1] = __uint_as_float(raw.x & 0xffff0000u);
+      f[2] = __uint_as_float(raw.y << 16); f[3] = __uint_as_float(raw.y & 0xffff0000u);
+    } else {
+      const uint32_t raw = *reinterpret_cast<const uint32_t*>(v + d0);
+      f[0] = __uint_as_float(raw << 16); f[1] = __uint_as_float(raw & 0xffff0000u);
+    }
     if (w != nullptr) {
       float ss = 0.f;
 #pragma unroll
@@ -149,13 +160,19 @@ head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq
 #pragma unroll
       for (int e = 0; e < DPL; ++e) f[e] = __bfloat162float(__float2bfloat16(f[e] * inv * bf16_bits_to_float(w[d0 + e])));
     }
+    float r[DPL];
 #pragma unroll
     for (int e = 0; e < DPL; ++e) {
       const float other = __shfl_xor_sync(0xffffffffu, f[e], 16);        // dim d0 + e -/+ D/2
       const int i = (d0 + e) % half;
-      const float r = low ? f[e] * cs_s[i] - other * sn_s[i] : f[e] * cs_s[i] + other * sn_s[i];
-      const __nv_bfloat16 hb = __float2bfloat16(r);
-      v[d0 + e] = *reinterpret_cast<const uint16_t*>(&hb);
+      r[e] = low ? f[e] * cs_s[i] - other * sn_s[i] : f[e] * cs_s[i] + other * sn_s[i];
+    }
+    __nv_bfloat162 h01 = __floats2bfloat162_rn(r[0], r[1]);
+    if constexpr (DPL == 4) {
+      __nv_bfloat162 h23 = __floats2bfloat162_rn(r[2], r[3]);
+      *reinterpret_cast<uint2*>(v + d0) = make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
+    } else {
+      *reinterpret_cast<uint32_t*>(v + d0) = *reinterpret_cast<uint32_t*>(&h01);
     }
   }
 }
@@ -266,11 +283,13 @@ extern "C" relaxkv_status relaxkv_qk_norm_rope(void* q, void* k, int64_t n_rows,
   if (n_rows == 0) return RELAXKV_OK;
   if (n_rows > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int heads_per_block = (n_rows >= 2048) ? n_q_heads + n_kv_heads : 4;
+  const dim3 grid((unsigned)n_rows, (unsigned)((n_q_heads + n_kv_heads + heads_per_block - 1) / heads_per_block));
   if (head_dim == 128)
-    head_norm_rope_kernel<128><<<(unsigned)n_rows, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads,
+    head_norm_rope_kernel<128><<<grid, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads, heads_per_block,
         static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
   else
-    head_norm_rope_kernel<64><<<(unsigned)n_rows, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads,
+    head_norm_rope_kernel<64><<<grid, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads, heads_per_block,
         static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
   return launch_ok();
 }

@@ -58,11 +58,10 @@ class LayerLoop:
             rec("norm", lambda: B.relaxkv_rmsnorm(h, w["w_in_norm"], x, blk.eps))
             rec("qkv_proj", lambda: (B.relaxkv_linear(x, w["wq"], q.view(n, -1)), B.relaxkv_linear(x, w["wk"], k.view(n, -1)),
                                      B.relaxkv_linear(x, w["wv"], v.view(n, -1))))
-            if "w_q_norm" in w:                       # per-head RMSNorm of the projected queries and keys, in place
-                rec("norm", lambda: (B.relaxkv_rmsnorm(q.view(-1, D), w["w_q_norm"], q.view(-1, D), blk.eps),
-                                     B.relaxkv_rmsnorm(k.view(-1, D), w["w_k_norm"], k.view(-1, D), blk.eps)))
+            # per-head RMSNorm of the projected queries and keys (models that have one) and the rotary embedding at the
+            # targets' original positions: one pass over q and k
             rec("rope", lambda: (B.relaxkv_target_positions(s.shape, s.u_pos, s.u_cu, s.r_rank, s.r_cu_layer(l), n_r[l], pos),
-                                 B.relaxkv_rope(q, pos, blk.rope_theta), B.relaxkv_rope(k, pos, blk.rope_theta)))
+                                 B.relaxkv_qk_norm_rope(q, k, pos, blk.rope_theta, w.get("w_q_norm"), w.get("w_k_norm"), blk.eps)))
             rec("attention", lambda: s.attention(l, caches[l], q, k, v, o, n_r[l], n_u))
             rec("scatter", lambda: s.scatter(l, caches[l], k, v, n_r[l]))
             rec("o_proj", lambda: B.relaxkv_linear(o.view(n, -1), w["wo"], a, residual=h))
