@@ -16,6 +16,8 @@
 // When a call has too few query tiles to fill the GPU, grid.y splits every pair's context; the blocks leave
 // normalised partial results that combine_splits_kernel merges by their log-sum-exp.  The K/V tensor maps
 // cover either the materialised mixed context (the repair calls) or the cache itself (relaxkv_cache_attention).
+// Calls over short gathered contexts (at most 128 key tiles, one split) take attention_persist_kernel below: one
+// block per SM walks the same list of (tile pair, KV head) items and overlaps each turn-over with its neighbours.
 // Every wait is bounded; an expired wait raises the block's abort flag, records RELAXKV_ERR_TIMEOUT in the
 // device status word and the block tears down normally.
 #include "attention_common.cuh"
