@@ -433,6 +433,9 @@ relaxkv_status relaxkv_sparse_ctx_attention_simt(
  *   out  device bf16 [n_target_rows, H, D]; lse_out optional device fp32 [H, n_target_rows]
  * The cache must hold max_b(h_req_token_offset[b] + h_ctx_len[b]) token rows.  Errors as for
  * relaxkv_sparse_ctx_attention (positions out of range are reported in the device status word).
+ * When every h_max_targets[b] <= 1 (a decode step) the call takes a streaming kernel instead of the 128-row tensor-core
+ * tiles: K and V tiles through a TMA ring, the request's few query heads in one warp-level MMA fragment, the context
+ * split over one wave of thread blocks and merged in a fixed order.
  */
 relaxkv_status relaxkv_cache_attention(
     const relaxkv_shape* shape, const relaxkv_cache_view* cache, const void* q_new,

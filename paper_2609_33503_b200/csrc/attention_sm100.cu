@@ -21,6 +21,7 @@
 // Every wait is bounded; an expired wait raises the block's abort flag, records RELAXKV_ERR_TIMEOUT in the
 // device status word and the block tears down normally.
 #include "attention_common.cuh"
+#include "decode_attention.cuh"
 #include "sm100_ptx.cuh"
 #include <algorithm>
 #include <atomic>
@@ -1033,31 +1034,54 @@ __global__ void wait_timeout_probe_kernel(DeviceStatus* st) {
   }
 }
 
+constexpr int kCombineThreads = 128;
+constexpr int kMaxCombineSplits = 1024;       // four warps x 4 KB of weights
+
 // Merges the partial results of a context split: out = sum_s w_s O_s / sum_s w_s with w_s = exp(lse_s - max lse).
 // One warp per (target row, query head); rows past the true target count are left alone.
-__global__ void combine_splits_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits,
-                                      long long n_target_rows, int H, int D, const int* __restrict__ r_cu, int n_req,
-                                      uint16_t* __restrict__ out, float* __restrict__ lse_out) {
-  const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(kCombineThreads)
+combine_splits_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits,
+                      long long n_target_rows, int H, int D, const int* __restrict__ r_cu, int n_req,
+                      uint16_t* __restrict__ out, float* __restrict__ lse_out) {
+  // the splits' weights of this warp's (row, head): the lanes fetch the log-sum-exps side by side (a serial walk over
+  // the splits would pay one memory latency per split), the sums below still run in split order
+  __shared__ float wgt_s[kCombineThreads / 32][kMaxCombineSplits];
+  const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long w = (long long)blockIdx.x * (kCombineThreads / 32) + wib;
   const long long rows_true = min((long long)(r_cu[n_req] - r_cu[0]), n_target_rows);
   if (w >= rows_true * H) return;
   const long long row = w / H;
   const int h = (int)(w - row * H);
   float mx = -INFINITY;
-  for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, part_lse[((long long)sp * n_target_rows + row) * H + h]);
+  for (int sp = lane; sp < n_splits; sp += 32) {
+    const float l = part_lse[((long long)sp * n_target_rows + row) * H + h];
+    wgt_s[wib][sp] = l;
+    mx = fmaxf(mx, l);
+  }
+  mx = warp_reduce_max(mx);
+  __syncwarp();
+  for (int sp = lane; sp < n_splits; sp += 32) {
+    const float l = wgt_s[wib][sp];
+    wgt_s[wib][sp] = (l == -INFINITY || mx == -INFINITY) ? 0.f : __expf(l - mx);
+  }
+  __syncwarp();
   const int per = D / 32;                       // 2 or 4 consecutive floats per lane
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   float den = 0.f;
-  if (mx > -INFINITY) {
-    for (int sp = 0; sp < n_splits; ++sp) {     // fixed order: reproducible
-      const long long slot = ((long long)sp * n_target_rows + row) * H + h;
-      const float l = part_lse[slot];
-      if (l == -INFINITY) continue;
-      const float wgt = __expf(l - mx);
-      den += wgt;
-      const float* o = part_o + slot * D + lane * per;
-      for (int e = 0; e < per; ++e) acc[e] += wgt * o[e];
+  const float* o = part_o + (row * H + h) * D + lane * per;
+  const long long sp_stride = n_target_rows * H * D;
+#pragma unroll 8
+  for (int sp = 0; sp < n_splits; ++sp) {       // fixed order: reproducible
+    const float wgt = wgt_s[wib][sp];
+    den += wgt;
+    const bool live = wgt > 0.f;                  // an empty split wrote no partial output: whatever is there is ignored
+    if (per == 4) {
+      const float4 v = *reinterpret_cast<const float4*>(o + sp * sp_stride);
+      acc[0] = fmaf(wgt, live ? v.x : 0.f, acc[0]); acc[1] = fmaf(wgt, live ? v.y : 0.f, acc[1]);
+      acc[2] = fmaf(wgt, live ? v.z : 0.f, acc[2]); acc[3] = fmaf(wgt, live ? v.w : 0.f, acc[3]);
+    } else {
+      const float2 v = *reinterpret_cast<const float2*>(o + sp * sp_stride);
+      acc[0] = fmaf(wgt, live ? v.x : 0.f, acc[0]); acc[1] = fmaf(wgt, live ? v.y : 0.f, acc[1]);
     }
   }
   const float inv = den > 0.f ? 1.f / den : 0.f;
@@ -1067,6 +1091,18 @@ __global__ void combine_splits_kernel(const float* __restrict__ part_o, const fl
     *reinterpret_cast<uint32_t*>(optr + e) = *reinterpret_cast<uint32_t*>(&h2);
   }
   if (lane == 0 && lse_out) lse_out[(long long)h * n_target_rows + row] = den > 0.f ? mx + logf(den) : -INFINITY;
+}
+
+relaxkv_status launch_combine_splits(const float* part_o, const float* part_lse, int n_splits, long long n_target_rows, int H,
+                                     int D, const int32_t* r_cu, int n_req, long long rows_bound, void* out, float* lse_out,
+                                     cudaStream_t stream) {
+  const long long warps = rows_bound * H;
+  if (warps <= 0) return RELAXKV_OK;
+  if (n_splits > kMaxCombineSplits) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
+  constexpr int wpb = kCombineThreads / 32;
+  combine_splits_kernel<<<(unsigned)((warps + wpb - 1) / wpb), kCombineThreads, 0, stream>>>(
+      part_o, part_lse, n_splits, n_target_rows, H, D, r_cu, n_req, static_cast<uint16_t*>(out), lse_out);
+  return launch_ok();
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -1184,10 +1220,8 @@ static relaxkv_status launch_attention(const relaxkv_shape* shape, int mode, Att
       u_pos, u_cu, r_rank, r_cu_layer, n_target_rows, static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st);
   relaxkv_status rc = launch_ok();
   if (rc != RELAXKV_OK || n_splits == 1) return rc;
-  const long long warps = plan.sum_targets * H;
-  combine_splits_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(
-      plan.split_o, plan.split_lse, (int)n_splits, n_target_rows, H, D, r_cu_layer, B, static_cast<uint16_t*>(out), lse_out);
-  return launch_ok();
+  return launch_combine_splits(plan.split_o, plan.split_lse, (int)n_splits, n_target_rows, H, D, r_cu_layer, B, plan.sum_targets,
+                               out, lse_out, stream);
 }
 
 }  // namespace relaxkv
@@ -1309,6 +1343,10 @@ extern "C" relaxkv_status relaxkv_cache_attention(
   plan.kv_token_stride_bytes = (unsigned long long)cache->token_stride * 2;
   plan.ctx_rows = cache_rows;
   plan.dense_ctx = 1;
+  // one target per request at most (a decode step): the streaming kernel
+  bool one_each = true;
+  for (int b = 0; b < shape->n_req; ++b) one_each = one_each && h_max_targets[b] <= 1;
+  if (one_each) return launch_decode_attention(shape, plan, q_new, tgt_pos, tgt_cu, n_target_rows, out, lse_out, stream);
   // lists: targets by position (their "rank" in the dense context), counts from tgt_cu; u_pos / u_cu are not read
   if (shape->head_dim == 128)
     return launch_attention<128>(shape, RELAXKV_CTX_UNION, plan, q_new, nullptr, nullptr, tgt_pos, tgt_cu, n_target_rows, out,

@@ -101,6 +101,38 @@ def test_persistent_form_at_32k_equals_the_one_shot_kernel():
     assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
 
 
+def test_decode_attention_at_32k():
+    """One decode token per request over 32K-token caches at the Qwen3-14B head layout, in the launch configuration the
+    time-to-first-token benchmark uses (automatic split: one wave of blocks): output and log-sum-exp against the oracle."""
+    from paper_2609_33503_b200 import binding as B
+    import oracle.relaxkv_oracle as orc
+    H, Hkv, D = 40, 8, 128
+    lens, pos = (32768, 20000), (32767, 12345)
+    offs = [0, 32768 + 64]
+    rows = offs[1] + lens[1] + 64
+    g = torch.Generator(device="cpu").manual_seed(21)
+    k_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    v_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    q = torch.randn(2, H, D, generator=g).to(torch.bfloat16).cuda()
+    shape = B.Shape(H, Hkv, D, list(lens), None, D ** -0.5)
+    ws = torch.empty(B.relaxkv_workspace_bytes(shape, 1) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.zeros_like(q)
+    lse = torch.zeros(H, 2, dtype=torch.float32, device="cuda")
+    B.relaxkv_cache_attention(shape, B.CacheView(k_all, v_all, offs), q, torch.tensor(pos, dtype=torch.int32).cuda(),
+                              torch.tensor([0, 1, 2], dtype=torch.int32).cuda(), [1, 1], out, ws, lse_out=lse)
+    st, detail = B.relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+    for b in range(2):
+        kb = inputs.bf16_bits(k_all[offs[b]:offs[b] + lens[b]].contiguous())
+        vb = inputs.bf16_bits(v_all[offs[b]:offs[b] + lens[b]].contiguous())
+        ref, ref_lse = orc.list_attention(kb, vb, inputs.bf16_bits(q[b:b + 1]), None, None, np.arange(lens[b]),
+                                          np.array([pos[b]], dtype=np.int32), D ** -0.5)
+        mx, mean = attention_errors(out[b:b + 1], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (b, mx, mean)
+        np.testing.assert_allclose(lse[:, b:b + 1].cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+
+
 def test_maximum_batch_of_64_requests():
     """The request table's limit (64 requests in one call) with ragged lengths from 1 token upwards:
     scores, anchors, sets, attention of every row, and the cache update against the oracle."""

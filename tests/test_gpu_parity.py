@@ -727,6 +727,68 @@ def test_cache_attention_of_query_rows_and_a_decode_step(head_major, n_splits):
     assert st == B().ERR_BAD_INDEX
 
 
+@pytest.mark.parametrize("H,Hkv,D", [(8, 8, 64), (12, 4, 128), (40, 8, 128), (32, 2, 64)], ids=["g1_d64", "g3_d128", "g5_d128", "g16_d64"])
+@pytest.mark.parametrize("n_splits,head_major", [(0, False), (1, True), (5, False)])
+def test_decode_attention_one_token_per_request(H, Hkv, D, n_splits, head_major):
+    """A decode step: at most one token per request attends to its cache prefix through the streaming kernel (TMA ring,
+    warp-level MMA fragments, split merge).  Five requests in one call - contexts of 1, 33, 129, 1000 and 2049 tokens,
+    the token's position anywhere in the request, one request without a token - with NaN / Inf in the rows between the
+    requests, against the oracle's explicit-list attention; then a position past the request's end and a second token
+    where the host promised one are reported, not read."""
+    lens = (1, 33, 129, 1000, 2049)
+    has = (1, 1, 0, 1, 1)
+    pos = (0, 32, 0, 700, 2048)
+    offs, rows = [], 0
+    for t in lens:
+        offs.append(rows); rows += t + 40                          # 40 rows that belong to nobody behind every request
+    g = torch.Generator(device="cpu").manual_seed(9)
+    k_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    v_all = torch.randn(rows, Hkv, D, generator=g).to(torch.bfloat16).cuda()
+    for o, t in zip(offs, lens):
+        k_all[o + t:o + t + 40] = float("nan")
+        v_all[o + t:o + t + 40:2] = float("nan")
+        v_all[o + t + 1:o + t + 40:2] = float("-inf")
+    if head_major:
+        k_all = k_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
+        v_all = v_all.permute(1, 0, 2).contiguous().permute(1, 0, 2)
+    n = sum(has)
+    q = torch.randn(n + 1, H, D, generator=g).to(torch.bfloat16).cuda()        # one spare row that must stay untouched
+    tgt_pos = torch.tensor([p for p, h in zip(pos, has) if h], dtype=torch.int32).cuda()
+    tgt_cu = torch.tensor(np.concatenate([[0], np.cumsum(has)]).astype(np.int32)).cuda()
+    shape = B().Shape(H, Hkv, D, list(lens), None, D ** -0.5, attention_ctx_splits=n_splits)
+    ws = torch.empty(B().relaxkv_workspace_bytes(shape, 1) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out = torch.full_like(q, 3.0)
+    lse = torch.zeros(H, n + 1, dtype=torch.float32, device="cuda")
+    view = B().CacheView(k_all, v_all, offs)
+    B().relaxkv_cache_attention(shape, view, q, tgt_pos, tgt_cu, [1] * len(lens), out, ws, lse_out=lse)   # loose bound for request 2
+    assert_status_ok()
+    row = 0
+    for b in range(len(lens)):
+        if not has[b]:
+            continue
+        kb = inputs.bf16_bits(k_all[offs[b]:offs[b] + lens[b]].contiguous())
+        vb = inputs.bf16_bits(v_all[offs[b]:offs[b] + lens[b]].contiguous())
+        ref, ref_lse = orc.list_attention(kb, vb, inputs.bf16_bits(q[row:row + 1]), None, None, np.arange(lens[b]),
+                                          np.array([pos[b]], dtype=np.int32), D ** -0.5)
+        mx, mean = attention_errors(out[row:row + 1], ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (b, mx, mean)
+        np.testing.assert_allclose(lse[:, row:row + 1].cpu().numpy().T, ref_lse, atol=2e-3, rtol=1e-4)
+        row += 1
+    assert torch.all(out[n] == 3.0)
+    bad = tgt_pos.clone()
+    bad[1] = lens[1]                                               # one past the end of request 1
+    B().relaxkv_cache_attention(shape, view, q, bad, tgt_cu, [1] * len(lens), out, ws)
+    st, _ = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX
+    two = torch.tensor([0, 1, 3, 3, 4, 5], dtype=torch.int32).cuda()            # request 1 brings two tokens
+    guard = torch.full((6, H, D), 3.0, dtype=torch.bfloat16, device="cuda")
+    B().relaxkv_cache_attention(shape, view, torch.cat([q, q])[:6].contiguous(), torch.tensor([0, 5, 6, 1, 2], dtype=torch.int32).cuda(),
+                                two, [1] * len(lens), guard, ws)
+    st, _ = B().relaxkv_read_device_status()
+    assert st == B().ERR_BAD_INDEX
+
+
 def _one_rank_group():
     """A process group of this one process on the GPU (NCCL): the all-reduce of the sharded path runs for real,
     over a single rank."""
