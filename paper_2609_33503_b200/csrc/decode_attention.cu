@@ -43,12 +43,6 @@ struct DecSmem {
   static constexpr int kDynamic = kTotal + 1024;
 };
 
-__device__ __forceinline__ void unpack8_bf16(const uint4& v, float* f) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(w[e] << 16); f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
-}
-
 __device__ __forceinline__ void ldmatrix_x4(uint32_t* r, uint32_t smem_addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr) : "memory");
@@ -71,9 +65,6 @@ decode_attention_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                         float scale_log2, uint16_t* __restrict__ out, float* __restrict__ lse_out, float* __restrict__ part_o,
                         float* __restrict__ part_lse, DeviceStatus* st) {
   using L = DecSmem<D>;
-  constexpr int DPL = D / 32;                       // head dims per lane in the P V phase
-  constexpr int kLanesPerRow = D / 8;               // lanes that cover one key row with 16-byte reads (16 or 8)
-  constexpr int kRowsPerLoad = 32 / kLanesPerRow;   // key rows one warp-wide load covers (2 or 4)
   const int G = H / Hkv;
   const int b = blockIdx.z, hd = blockIdx.y, split = blockIdx.x, n_splits = gridDim.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
