@@ -78,6 +78,26 @@ def test_linear_qkv_writes_the_three_projections(M, n_q, n_kv, K):
             assert torch.equal(one, out)
 
 
+@pytest.mark.parametrize("M,N,K,res", [(5, 8, 8, False), (17, 136, 72, True), (100, 1000, 520, True), (128, 5120, 1032, False),
+                                       (64, 264, 5120, True), (128, 19200, 64, False), (33, 2048, 17408, True)])
+def test_linear_of_a_few_rows(M, N, K, res):
+    """5 to 128 rows: 128 x 128 tiles whose K range is split over a thread-block cluster (1 to 8 blocks, by the
+    number of column tiles and K blocks) and summed through distributed shared memory; ragged N and K tails, a residual
+    that aliases the output, K shorter than two blocks per cluster member, more column tiles than SMs (19200 / 128 =
+    150: the large kernel takes that one); run twice: bit-identical (the partial sums are added in rank order)."""
+    x, w = rnd(M, K, seed=41), rnd(N, K, scale=K ** -0.5, seed=42)
+    r = rnd(M, N, seed=43) if res else None
+    y = r.clone() if res else torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    B().relaxkv_linear(x, w, y, residual=y if res else None)
+    st, detail = B().relaxkv_read_device_status()
+    assert st == 0, (st, detail)
+    ref = blk.linear(blk.f64(bits(x)), blk.f64(bits(w)), blk.f64(bits(r)) if res else None)
+    close(y, ref, abs_floor=4e-3)
+    y2 = r.clone() if res else torch.empty_like(y)
+    B().relaxkv_linear(x, w, y2, residual=y2 if res else None)
+    assert torch.equal(y, y2)
+
+
 def test_linear_at_the_benchmark_shapes():
     """The projections at the sizes the repair loop runs them for the 32K Qwen3-14B-shaped stack: 18 000 active rows
     through a 5120 -> 5120 projection with residual (SM pairs) and the fused gate/up projection of 5120 -> 2 x 17408 on
