@@ -113,6 +113,32 @@ def test_bad_arguments_are_rejected_on_the_host():
                                  i32([200]), FAKE, FAKE, I64(100), NULL) == B.ERR_INVALID_ARG     # too few rows
 
 
+def test_block_work_calls_reject_bad_arguments_on_the_host():
+    """The projections and the fused norm + rotary call check pointers, alignment and shapes before any launch."""
+    lib = B.lib()
+    F32 = ctypes.c_float
+    lin = lambda x, w, y, rows, n_out, n_in, res=NULL: lib.relaxkv_linear(x, w, res, y, I64(rows), n_out, n_in, NULL)
+    assert lin(NULL, FAKE, FAKE, 4, 64, 64) == B.ERR_INVALID_ARG
+    assert lin(FAKE, FAKE, ctypes.c_void_p(0x10002), 4, 64, 64) == B.ERR_INVALID_ARG          # output not 16-byte aligned
+    assert lin(FAKE, FAKE, FAKE, 4, 60, 64) == B.ERR_UNSUPPORTED_SHAPE                        # widths are multiples of 8
+    assert lin(FAKE, FAKE, FAKE, -1, 64, 64) == B.ERR_UNSUPPORTED_SHAPE
+    assert lin(FAKE, FAKE, FAKE, 0, 64, 64) == B.OK                                           # nothing to do
+    qkv = lambda x, w, q, k, v, rows, n_q, n_kv, n_in: lib.relaxkv_linear_qkv(x, w, q, k, v, I64(rows), n_q, n_kv, n_in, NULL)
+    assert qkv(FAKE, FAKE, FAKE, NULL, FAKE, 4, 64, 16, 64) == B.ERR_INVALID_ARG
+    assert qkv(FAKE, ctypes.c_void_p(0x10008), FAKE, FAKE, FAKE, 4, 64, 16, 64) == B.ERR_INVALID_ARG
+    assert qkv(FAKE, FAKE, FAKE, FAKE, FAKE, 4, 64, 12, 64) == B.ERR_UNSUPPORTED_SHAPE
+    assert qkv(FAKE, FAKE, FAKE, FAKE, FAKE, 0, 64, 16, 64) == B.OK
+    assert lib.relaxkv_linear_swiglu(FAKE, FAKE, FAKE, I64(4), 100, 64, NULL) == B.ERR_UNSUPPORTED_SHAPE   # 128-feature blocks
+    nr = lambda q, k, rows, hq, hkv, d, wq, wk, eps, pos, theta: lib.relaxkv_qk_norm_rope(
+        q, k, I64(rows), hq, hkv, d, wq, wk, F32(eps), pos, F32(theta), NULL)
+    assert nr(FAKE, NULL, 4, 8, 2, 128, NULL, NULL, 1e-6, FAKE, 1e6) == B.ERR_INVALID_ARG
+    assert nr(FAKE, FAKE, 4, 8, 2, 128, FAKE, NULL, 1e-6, FAKE, 1e6) == B.ERR_INVALID_ARG     # one norm weight without the other
+    assert nr(FAKE, FAKE, 4, 8, 2, 128, NULL, NULL, 1e-6, NULL, 1e6) == B.ERR_INVALID_ARG     # no positions
+    assert nr(FAKE, FAKE, 4, 8, 2, 128, NULL, NULL, 1e-6, FAKE, 1.0) == B.ERR_INVALID_ARG     # theta must exceed 1
+    assert nr(FAKE, FAKE, 4, 8, 2, 96, NULL, NULL, 1e-6, FAKE, 1e6) == B.ERR_UNSUPPORTED_SHAPE
+    assert nr(FAKE, FAKE, 0, 8, 2, 128, NULL, NULL, 1e-6, FAKE, 1e6) == B.OK
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/librelaxkv.so")
