@@ -384,6 +384,15 @@ def test_edge_sizes(ctx, q, ratio):
         for full_prefix in (False, True):
             out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
             check_attention(case, l, out, lse, full_prefix)
+    # the same sizes through the persistent form: two blocks walk every item (one-tile contexts, items without work)
+    s.shape.set_tuning(attention_ctx_splits=1, attention_persistent=1, attention_grid_blocks=2)
+    try:
+        for l in range(w.n_layers):
+            for full_prefix in (False, True):
+                out, lse = run_attention(case, s, l, B().CTX_FULL_PREFIX if full_prefix else B().CTX_UNION, simt=False)
+                check_attention(case, l, out, lse, full_prefix)
+    finally:
+        s.shape.set_tuning()
 
 
 def test_loose_host_bounds_give_the_same_result(case):
