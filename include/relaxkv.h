@@ -451,6 +451,19 @@ relaxkv_status relaxkv_cache_attention(
 relaxkv_status relaxkv_debug_wait_timeout(relaxkv_stream stream);
 
 /*
+ * Chained launches.  The short kernels of a decode step (RMSNorm, norm + rotary and the cache append
+ * of at most 8 rows, the one- to four-row projections, the one-token attention and its merge) are
+ * launched with CUDA's programmatic stream serialization: the next kernel's blocks become resident
+ * while the current kernel finishes, request the head of their weights into L2 (weights depend on
+ * no earlier kernel) and then wait, inside the kernel, until every earlier kernel of the stream has
+ * completed and its writes are visible.  Results are identical to plain
+ * launches; stream order as the caller sees it is unchanged; the launches can be captured into a
+ * CUDA graph.  relaxkv_set_chained_launch(0) switches to plain launches for the whole process
+ * (1 = chained, the default) and returns the previous setting; it affects calls made after it.
+ */
+int32_t relaxkv_set_chained_launch(int32_t on);
+
+/*
  * Synchronises `stream`, copies the device status word (a relaxkv_status: RELAXKV_OK,
  * RELAXKV_ERR_BAD_INDEX or RELAXKV_ERR_TIMEOUT, the first problem recorded wins) to
  * *h_status_out and clears it.  h_detail_out (NULL or host int32[4]) receives where it happened:

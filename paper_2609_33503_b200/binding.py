@@ -26,7 +26,7 @@ ENTRY_POINTS = (
     "relaxkv_build_active_sets_static", "relaxkv_debug_wait_timeout",
     "relaxkv_list_attention", "relaxkv_cache_attention",
     "relaxkv_scatter_kv_lists", "relaxkv_mean_scores", "relaxkv_scale_scores", "relaxkv_query_prefill_attention", "relaxkv_rmsnorm", "relaxkv_linear", "relaxkv_linear_qkv", "relaxkv_linear_swiglu", "relaxkv_rope", "relaxkv_qk_norm_rope",
-    "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows",
+    "relaxkv_swiglu", "relaxkv_target_positions", "relaxkv_carry_rows", "relaxkv_set_chained_launch",
 )
 
 
@@ -78,6 +78,12 @@ def lib() -> ctypes.CDLL:
 
 def status_string(status: int) -> str:
     return lib().relaxkv_status_string(int(status)).decode()
+
+
+def relaxkv_set_chained_launch(on: bool) -> bool:
+    """Chained (programmatic dependent) launches of the short kernels on or off, process-wide; returns the previous
+    setting."""
+    return bool(lib().relaxkv_set_chained_launch(1 if on else 0))
 
 
 def _check(status: int, where: str) -> None:

@@ -35,9 +35,16 @@ int sm_count_of_current_device() {
   return n;
 }
 
+static std::atomic<int> g_chained_launch{1};
+bool chained_launch_enabled() { return g_chained_launch.load(std::memory_order_relaxed) != 0; }
+
 }  // namespace relaxkv
 
 using namespace relaxkv;
+
+extern "C" int32_t relaxkv_set_chained_launch(int32_t on) {
+  return g_chained_launch.exchange(on ? 1 : 0, std::memory_order_relaxed);
+}
 
 extern "C" const char* relaxkv_status_string(int32_t status) {
   switch (status) {

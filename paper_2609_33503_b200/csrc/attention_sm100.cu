@@ -1048,6 +1048,8 @@ combine_splits_kernel(const float* __restrict__ part_o, const float* __restrict_
   __shared__ float wgt_s[kCombineThreads / 32][kMaxCombineSplits];
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long w = (long long)blockIdx.x * (kCombineThreads / 32) + wib;
+  griddep_launch();
+  griddep_wait();                               // the partial results come from the kernel before
   const long long rows_true = min((long long)(r_cu[n_req] - r_cu[0]), n_target_rows);
   if (w >= rows_true * H) return;
   const long long row = w / H;
@@ -1100,9 +1102,8 @@ relaxkv_status launch_combine_splits(const float* part_o, const float* part_lse,
   if (warps <= 0) return RELAXKV_OK;
   if (n_splits > kMaxCombineSplits) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   constexpr int wpb = kCombineThreads / 32;
-  combine_splits_kernel<<<(unsigned)((warps + wpb - 1) / wpb), kCombineThreads, 0, stream>>>(
-      part_o, part_lse, n_splits, n_target_rows, H, D, r_cu, n_req, static_cast<uint16_t*>(out), lse_out);
-  return launch_ok();
+  return cuda_ok(launch_chained(n_target_rows <= kChainedMaxRows, combine_splits_kernel, (unsigned)((warps + wpb - 1) / wpb), kCombineThreads, 0, stream, part_o,
+                                part_lse, n_splits, (long long)n_target_rows, H, D, r_cu, n_req, static_cast<uint16_t*>(out), lse_out));
 }
 
 // ---- host side ---------------------------------------------------------------------------------------

@@ -68,6 +68,8 @@ decode_attention_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const int G = H / Hkv;
   const int b = blockIdx.z, hd = blockIdx.y, split = blockIdx.x, n_splits = gridDim.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  griddep_launch();
+  griddep_wait();                          // q, the lists and the newest cache row come from the kernels before
   const int nr = tgt_cu[b + 1] - tgt_cu[b];
   if (nr <= 0) return;
   const long long row = (long long)tgt_cu[b] - tgt_cu[0];
@@ -312,10 +314,9 @@ static relaxkv_status launch_g(const CUtensorMap& tm_k, const CUtensorMap& tm_v,
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DecSmem<D>::kDynamic) != cudaSuccess) return RELAXKV_ERR_CUDA;
     attr_done[dev].store(1, std::memory_order_release);
   }
-  kern<<<grid, kDecThreads, DecSmem<D>::kDynamic, stream>>>(tm_k, tm_v, plan.rt, static_cast<const uint16_t*>(q), tgt_pos, tgt_cu,
-                                                           n_target_rows, H, Hkv, scale_log2, static_cast<uint16_t*>(out), lse_out,
-                                                           plan.split_o, plan.split_lse, st);
-  return launch_ok();
+  return cuda_ok(launch_chained(true, kern, grid, kDecThreads, DecSmem<D>::kDynamic, stream, tm_k, tm_v, plan.rt,
+                                static_cast<const uint16_t*>(q), tgt_pos, tgt_cu, (long long)n_target_rows, H, Hkv, scale_log2,
+                                static_cast<uint16_t*>(out), lse_out, plan.split_o, plan.split_lse, st));
 }
 
 template <int D>

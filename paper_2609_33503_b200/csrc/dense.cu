@@ -26,6 +26,8 @@ rmsnorm_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, u
   const long long row = blockIdx.x;
   const uint16_t* xr = x + row * C;
   float ss = 0.f;
+  griddep_launch();
+  griddep_wait();
   for (int i = threadIdx.x * 8; i < C; i += 256 * 8) {
     float f[8];
     unpack8(__ldg(reinterpret_cast<const uint4*>(xr + i)), f);
@@ -57,6 +59,8 @@ rmsnorm_short_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
                      int C, float eps) {
   const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
+  griddep_launch();
+  griddep_wait();
   if (row >= rows) return;
   const bool mine = lane * 8 < C;
   float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -126,6 +130,8 @@ head_norm_rope_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, int Hq
   constexpr int DPL = D / 32, half = D / 2;
   __shared__ float cs_s[half], sn_s[half];
   const long long row = blockIdx.x;
+  griddep_launch();
+  griddep_wait();                                             // the positions may come from the kernel before
   if (threadIdx.x < half) {
     const int i = threadIdx.x;
     const double inv_freq = exp2(-(double)log2_theta * (2.0 * i / D));
@@ -251,14 +257,14 @@ extern "C" relaxkv_status relaxkv_rmsnorm(const void* x, const void* weight, voi
   if (n_cols <= 256) {
     const long long blocks = (n_rows * 32 + 255) / 256;
     if (blocks > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
-    rmsnorm_short_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(y), n_rows, n_cols, eps);
-    return launch_ok();
+    return cuda_ok(launch_chained(n_rows <= kChainedMaxRows, rmsnorm_short_kernel, (unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream),
+                                  static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight),
+                                  static_cast<uint16_t*>(y), (long long)n_rows, n_cols, eps));
   }
   if (n_rows > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
-  rmsnorm_kernel<<<(unsigned)n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(y), n_cols, eps);
-  return launch_ok();
+  return cuda_ok(launch_chained(n_rows <= kChainedMaxRows, rmsnorm_kernel, (unsigned)n_rows, 256, 0, static_cast<cudaStream_t>(stream),
+                                static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(weight),
+                                static_cast<uint16_t*>(y), n_cols, eps));
 }
 
 extern "C" relaxkv_status relaxkv_rope(void* x, int64_t n_rows, int32_t n_heads, int32_t head_dim, const int32_t* positions,
@@ -285,13 +291,16 @@ extern "C" relaxkv_status relaxkv_qk_norm_rope(void* q, void* k, int64_t n_rows,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int heads_per_block = (n_rows >= 2048) ? n_q_heads + n_kv_heads : 4;
   const dim3 grid((unsigned)n_rows, (unsigned)((n_q_heads + n_kv_heads + heads_per_block - 1) / heads_per_block));
+  uint16_t* qp = static_cast<uint16_t*>(q);
+  uint16_t* kp = static_cast<uint16_t*>(k);
+  const uint16_t* wq = static_cast<const uint16_t*>(w_q_norm);
+  const uint16_t* wk = static_cast<const uint16_t*>(w_k_norm);
+  const float log2_theta = log2f(theta);
   if (head_dim == 128)
-    head_norm_rope_kernel<128><<<grid, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads, heads_per_block,
-        static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
-  else
-    head_norm_rope_kernel<64><<<grid, 128, 0, st>>>(static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), n_q_heads, n_kv_heads, heads_per_block,
-        static_cast<const uint16_t*>(w_q_norm), static_cast<const uint16_t*>(w_k_norm), eps, positions, log2f(theta));
-  return launch_ok();
+    return cuda_ok(launch_chained(n_rows <= kChainedMaxRows, head_norm_rope_kernel<128>, grid, 128, 0, st, qp, kp, n_q_heads, n_kv_heads, heads_per_block,
+                                  wq, wk, eps, positions, log2_theta));
+  return cuda_ok(launch_chained(n_rows <= kChainedMaxRows, head_norm_rope_kernel<64>, grid, 128, 0, st, qp, kp, n_q_heads, n_kv_heads, heads_per_block,
+                                wq, wk, eps, positions, log2_theta));
 }
 
 extern "C" relaxkv_status relaxkv_swiglu(const void* gate_up, void* out, int64_t n_rows, int32_t n_inter, relaxkv_stream stream) {

@@ -245,6 +245,8 @@ scatter_kv_kernel(ReqTable rt, int n_kv_heads, int head_dim,
   const int B = rt.n_req;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long y0 = ((long long)blockIdx.x * kMoveWarps + warp) * rows_per_warp;
+  griddep_launch();
+  griddep_wait();                              // the rows and the index lists come from earlier kernels
   if (y0 >= rt.tile_cu[B]) return;             // rt.tile_cu = prefix of the host bounds on |R_{l,b}|
   const uint32_t bar = smem_u32(&bars[warp]);
   if (lane == 0) { gave_up[warp] = 0; mbar_init(bar, 1); fence_barrier_init(); }
@@ -342,11 +344,10 @@ static relaxkv_status launch_scatter(const relaxkv_shape* shape, const ReqTable&
   const long long rows_per_block = (long long)kMoveWarps * rows_per_warp;
   const long long blocks = (total + rows_per_block - 1) / rows_per_block;
   RELAXKV_RANGE("scatter_kv_kernel");
-  scatter_kv_kernel<<<(unsigned)blocks, kMoveThreads, smem, stream>>>(
+  return cuda_ok(launch_chained(total <= kChainedMaxRows, scatter_kv_kernel, (unsigned)blocks, kMoveThreads, smem, stream,
       rt, shape->n_kv_heads, shape->head_dim, static_cast<uint16_t*>(cache->k), static_cast<uint16_t*>(cache->v),
-      cache->token_stride, cache->head_stride, static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new),
-      u_pos, u_cu, r_rank, r_cu, direct, rows_per_warp, st);
-  return launch_ok();
+      (long long)cache->token_stride, (long long)cache->head_stride, static_cast<const uint16_t*>(k_new),
+      static_cast<const uint16_t*>(v_new), u_pos, u_cu, r_rank, r_cu, direct, rows_per_warp, st));
 }
 
 }  // namespace relaxkv

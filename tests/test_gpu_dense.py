@@ -459,3 +459,73 @@ def test_query_pass_prefill_scores_and_first_decode_step():
         check_layer(l, h_tok, out, (1, 1), [c + q for c, q in zip(ctx, qn)],
                     [k_after[l][offs[b]:offs[b] + ctx[b] + qn[b]] for b in range(nb)],
                     [v_after[l][offs[b]:offs[b] + ctx[b] + qn[b]] for b in range(nb)], False)
+
+
+@pytest.mark.parametrize("graph", [False, True], ids=["eager", "graph"])
+def test_decode_step_with_chained_launches_equals_plain_launches(graph):
+    """The few-row kernels of a decode step are launched with programmatic stream serialization (each kernel's blocks
+    become resident while its predecessor finishes and wait inside the kernel for it).  Same bits as plain launches:
+    logits of three decode steps in a row and the K/V rows they append, eagerly and replayed from a CUDA graph."""
+    from paper_2609_33503_b200.query_pass import QueryPass
+    H, Hkv, D = 8, 2, 128
+    ctx, qn = (700, 1300, 90), (1, 1, 1)
+    blkshape = inputs.BlockShape(hidden=2048, inter=4096, rope_theta=1.0e6, eps=1.0e-6, qk_norm=True)
+    w = inputs.Workload("chained", 3, H, Hkv, D, 64, ctx, qn, 0.15, base_seed=23)
+    L, nb, vocab, steps = 3, 3, 3000, 3
+    room = [c + q + steps for c, q in zip(ctx, qn)]
+    offs = [0, room[0], room[0] + room[1]]
+    weights = [inputs.block_weights(w, blkshape, l, "cuda") for l in range(L)]
+    w_final, w_head = rnd(blkshape.hidden, seed=41), rnd(vocab, blkshape.hidden, scale=blkshape.hidden ** -0.5, seed=42)
+    h_tok = rnd(nb, blkshape.hidden, seed=51)
+
+    def run(chained):
+        prev = B().relaxkv_set_chained_launch(chained)
+        try:
+            views, ks = [], []
+            for l in range(L):
+                k_all = torch.zeros(sum(room), Hkv, D, dtype=torch.bfloat16, device="cuda")
+                v_all = torch.zeros_like(k_all)
+                for b in range(nb):
+                    _, k, v = inputs.layer_qkv(w, l, b, "cuda")
+                    k_all[offs[b]:offs[b] + ctx[b]], v_all[offs[b]:offs[b] + ctx[b]] = k, v
+                ks.append((k_all, v_all))
+                views.append(B().CacheView(k_all, v_all, offs))
+            qp = QueryPass(H, Hkv, D, ctx, qn, blkshape, extra_tokens=steps)
+            logits = [torch.zeros(nb, vocab, dtype=torch.bfloat16, device="cuda") for _ in range(steps)]
+            for s in range(steps):
+                qp.decode_positions(s)
+
+            def all_steps():
+                for s in range(steps):
+                    qp.output_head(qp.decode(h_tok, weights, views, step=s), w_final, w_head, logits[s])
+            if graph:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    all_steps()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        all_steps()
+                torch.cuda.current_stream().wait_stream(side)
+                for lg in logits:
+                    lg.zero_()
+                g.replay()
+            else:
+                all_steps()
+            torch.cuda.synchronize()
+            st, detail = B().relaxkv_read_device_status()
+            assert st == 0, (st, detail)
+            return [lg.clone() for lg in logits], [(k.clone(), v.clone()) for k, v in ks]
+        finally:
+            B().relaxkv_set_chained_launch(prev)
+
+    plain, chained = run(False), run(True)
+    for s in range(steps):
+        assert torch.isfinite(plain[0][s].float()).all() and plain[0][s].float().abs().max() > 0
+        assert torch.equal(plain[0][s], chained[0][s]), s
+    for (k0, v0), (k1, v1) in zip(plain[1], chained[1]):
+        assert torch.equal(k0, k1) and torch.equal(v0, v1)
+    # the appended rows are where they belong: position T_c + Q_b + step of every request is no longer zero
+    for b in range(nb):
+        for s in range(steps):
+            assert plain[1][0][0][offs[b] + ctx[b] + qn[b] + s].float().abs().max() > 0
