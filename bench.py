@@ -1014,7 +1014,10 @@ def run_ttft(args):
            "decode_step": {"us": round(phase["decode_step"] * 1e3, 1), "weight_bytes": int(weight_bytes),
                            "weights_gbs": round(weight_bytes / (phase["decode_step"] * 1e-3) / 1e9, 1),
                            "frac_hbm": round(weight_bytes / (phase["decode_step"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
-                           "note": "bytes = every block weight and the output head once; K/V reads (2 x 40 x 67 MB) not counted"},
+                           "kv_bytes_not_counted": int(2 * L * (T + Q) * w.n_kv_heads * w.head_dim * 2),
+                           "launches": "few-row kernels chained (programmatic stream serialization)",
+                           "note": "bytes = every block weight and the output head once; the K/V reads of the step's "
+                                   "attention are listed beside it, not counted"},
            "clocks": clocks}
     print(json.dumps(out))
 
