@@ -139,6 +139,14 @@ def test_block_work_calls_reject_bad_arguments_on_the_host():
     assert nr(FAKE, FAKE, 0, 8, 2, 128, NULL, NULL, 1e-6, FAKE, 1e6) == B.OK
 
 
+def test_chained_launch_switch_is_host_state_only():
+    """relaxkv_set_chained_launch returns the previous setting and launches nothing (chained is the default)."""
+    assert B.relaxkv_set_chained_launch(False) is True
+    assert B.relaxkv_set_chained_launch(False) is False
+    assert B.relaxkv_set_chained_launch(True) is False
+    assert B.relaxkv_set_chained_launch(True) is True
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/librelaxkv.so")
