@@ -359,7 +359,8 @@ relaxkv_status relaxkv_linear(const void* x, const void* weight, const void* res
  * w_qkv [n_q + 2 n_kv, n_in] = the rows of Wq, then Wk, then Wv (stacked once when the weights are loaded).
  * x [n_rows, n_in]; q [n_rows, n_q], k and v [n_rows, n_kv]: three separate row-major buffers.  Same arithmetic per
  * output element as relaxkv_linear.  Up to 128 rows (a decode token, the query's own tokens) this is ONE kernel that
- * streams the stacked matrix once; for more rows it runs the three projections one after the other.
+ * streams the stacked matrix once; for more rows it is one large GEMM whose epilogue writes the three buffers when
+ * n_q and n_kv are multiples of 32, else the three projections one after the other.
  * n_q, n_kv, n_in multiples of 8. */
 relaxkv_status relaxkv_linear_qkv(const void* x, const void* w_qkv, void* q, void* k, void* v, int64_t n_rows,
                                   int32_t n_q, int32_t n_kv, int32_t n_in, relaxkv_stream stream);

@@ -24,10 +24,26 @@ constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;
 constexpr int kGemmBars = 2 * kGemmStages + 4;           // full, empty per stage; accumulator full, empty x 2
 constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 8 * kGemmBars + 16 + 1024;
 
+// Output columns split into up to three buffers of their own (the stacked Q/K/V projection): segment i = columns
+// [col0[i], col0[i + 1]) goes to the row-major buffer y[i] of that width.  n == 0: one buffer (the kernel's y).  The
+// boundaries are multiples of 32, the width of an epilogue chunk.
+struct GemmSegs {
+  uint16_t* y[3];
+  int col0[4];
+  int n;
+};
+// where the 32-column chunk that starts at output column col0 of `row` goes: base pointer of its first element
+__device__ __forceinline__ uint16_t* chunk_ptr(const GemmSegs& segs, uint16_t* y, long long row, int N, int col0) {
+  if (segs.n == 0) return y + row * N + col0;
+  int sg = 0;
+  while (sg + 1 < segs.n && col0 >= segs.col0[sg + 1]) ++sg;
+  return segs.y[sg] + row * (segs.col0[sg + 1] - segs.col0[sg]) + (col0 - segs.col0[sg]);
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   long long M, int N, int K, uint16_t* __restrict__ y, const uint16_t* __restrict__ residual,
-                  int swiglu, DeviceStatus* st) {
+                  int swiglu, const __grid_constant__ GemmSegs segs, DeviceStatus* st) {
   const int tiles_m = (int)((M + kGemmBM - 1) / kGemmBM), tiles_n = (N + kGemmBN - 1) / kGemmBN;
   const long long n_tiles = (long long)tiles_m * tiles_n;
   if (*reinterpret_cast<volatile int*>(&st->status) == RELAXKV_ERR_TIMEOUT) return;
@@ -156,6 +172,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int col0 = tn * kGemmBN + c * 32;
         if (row < M && col0 < N) {
           const long long off = row * N + col0;
+          uint16_t* yc = chunk_ptr(segs, y, row, N, col0);
 #pragma unroll
           for (int i8 = 0; i8 < 32; i8 += 8) {
             if (col0 + i8 < N) {                                 // N is a multiple of 8
@@ -174,7 +191,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
                 w[e] = *reinterpret_cast<uint32_t*>(&h2);
               }
-              *reinterpret_cast<uint4*>(y + off + i8) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(yc + i8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
@@ -205,7 +222,7 @@ constexpr int kPairSmem = kPairStages * kPairStageBytes + 8 * kPairBarsTotal + 1
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   long long M, int N, int K, uint16_t* __restrict__ y, const uint16_t* __restrict__ residual,
-                  int swiglu, DeviceStatus* st) {
+                  int swiglu, const __grid_constant__ GemmSegs segs, DeviceStatus* st) {
   // a cluster of two CTAs computes 256 x 256 output tiles: CTA rank r holds rows [128 r, 128 r + 128) of the tile's A
   // rows and of its B rows (= output columns), the leader's MMA thread drives both SMs (M = 256), every CTA drains
   // its own 128 x 256 accumulator.  tiles_m counts 256-row tiles here.  (No early exit after a timeout: the two
@@ -355,6 +372,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
         const int col0 = tn * kGemmBN + c * 32;
         if (row < M && col0 < N) {
           const long long off = row * N + col0;
+          uint16_t* yc = chunk_ptr(segs, y, row, N, col0);
 #pragma unroll
           for (int i8 = 0; i8 < 32; i8 += 8) {
             if (col0 + i8 < N) {                                 // N is a multiple of 8
@@ -373,7 +391,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
                 w[e] = *reinterpret_cast<uint32_t*>(&h2);
               }
-              *reinterpret_cast<uint4*>(y + off + i8) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(yc + i8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
@@ -400,7 +418,10 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 using namespace relaxkv;
 
 static relaxkv_status launch_gemm(const void* x, const void* weight, const void* residual, void* y, int64_t n_rows,
-                                  int32_t n_out, int32_t n_in, int swiglu, relaxkv_stream stream_) {
+                                  int32_t n_out, int32_t n_in, int swiglu, relaxkv_stream stream_,
+                                  const GemmSegs* segs_in = nullptr) {
+  GemmSegs segs = {};
+  if (segs_in) segs = *segs_in;
   if (!x || !weight || !y || !aligned16(x) || !aligned16(weight) || !aligned16(y) || (residual && !aligned16(residual)))
     return RELAXKV_ERR_INVALID_ARG;
   if (n_rows < 0 || n_out < 8 || n_in < 8 || (n_out % 8) || (n_in % 8)) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
@@ -466,14 +487,14 @@ static relaxkv_status launch_gemm(const void* x, const void* weight, const void*
     }
     const long long clusters = std::min<long long>(tiles_m2 * tiles_n, n_clusters);
     gemm_pair_sm100_kernel<<<(unsigned)(2 * clusters), kGemmThreads, kPairSmem, static_cast<cudaStream_t>(stream_)>>>(
-        tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, st);
+        tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, segs, st);
     return launch_ok();
   }
   const long long tiles_m = (n_rows + kGemmBM - 1) / kGemmBM;
   if (tiles_m * tiles_n > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   const long long grid = std::min<long long>(tiles_m * tiles_n, sms);     // persistent: one CTA per SM
   gemm_sm100_kernel<<<(unsigned)grid, kGemmThreads, kGemmSmem, static_cast<cudaStream_t>(stream_)>>>(
-      tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, st);
+      tm_a, tm_b, n_rows, n_out, n_in, static_cast<uint16_t*>(y), static_cast<const uint16_t*>(residual), swiglu, segs, st);
   return launch_ok();
 }
 
@@ -506,7 +527,16 @@ extern "C" relaxkv_status relaxkv_linear_qkv(const void* x, const void* w_qkv, v
     outs.n = 3;
     return launch_gemm_skinny(x, w_qkv, outs, (int)n_rows, n_out, n_in, stream);
   }
-  // many rows: the three projections one after the other (each is at the tensor peak on its own)
+  // many rows: one GEMM over the stacked matrix whose epilogue writes the three buffers (the K and V projections alone
+  // have four 256-column tiles each and leave the last wave of SM pairs half empty) ...
+  if (n_q % 32 == 0 && n_kv % 32 == 0) {
+    GemmSegs segs = {};
+    segs.y[0] = static_cast<uint16_t*>(q); segs.y[1] = static_cast<uint16_t*>(k); segs.y[2] = static_cast<uint16_t*>(v);
+    segs.col0[0] = 0; segs.col0[1] = n_q; segs.col0[2] = n_q + n_kv; segs.col0[3] = n_out;
+    segs.n = 3;
+    return launch_gemm(x, w_qkv, nullptr, q, n_rows, n_out, n_in, 0, stream_, &segs);
+  }
+  // ... unless a boundary falls inside a 32-column chunk of the epilogue: then the three projections one after the other
   const uint16_t* w = static_cast<const uint16_t*>(w_qkv);
   relaxkv_status rc = launch_gemm(x, w, nullptr, q, n_rows, n_q, n_in, 0, stream_);
   if (rc == RELAXKV_OK) rc = launch_gemm(x, w + (size_t)n_q * n_in, nullptr, k, n_rows, n_kv, n_in, 0, stream_);

@@ -56,8 +56,9 @@ class LayerLoop:
             x, a, q, k, v, o = self.x[:n], self.a[:n], self.q[:n], self.k[:n], self.v[:n], self.o[:n]
             gu, m, pos = self.gu[:n], self.m[:n], self.pos[:n]
             rec("norm", lambda: B.relaxkv_rmsnorm(h, w["w_in_norm"], x, blk.eps))
-            rec("qkv_proj", lambda: (B.relaxkv_linear(x, w["wq"], q.view(n, -1)), B.relaxkv_linear(x, w["wk"], k.view(n, -1)),
-                                     B.relaxkv_linear(x, w["wv"], v.view(n, -1))))
+            if "w_qkv" not in w:                            # weight-loading step, once per layer: [Wq; Wk; Wv] stacked
+                w["w_qkv"] = B.stack_qkv(w["wq"], w["wk"], w["wv"])
+            rec("qkv_proj", lambda: B.relaxkv_linear_qkv(x, w["w_qkv"], q.view(n, -1), k.view(n, -1), v.view(n, -1)))
             # per-head RMSNorm of the projected queries and keys (models that have one) and the rotary embedding at the
             # targets' original positions: one pass over q and k
             rec("rope", lambda: (B.relaxkv_target_positions(s.shape, s.u_pos, s.u_cu, s.r_rank, s.r_cu_layer(l), n_r[l], pos),

@@ -54,12 +54,14 @@ def _check_linear(M, N, K, res):
     torch.testing.assert_close(y.float(), (x.float() @ w.float().T + (r.float() if res else 0)), rtol=2e-2, atol=2e-2)
 
 
-@pytest.mark.parametrize("M", [1, 3, 5, 64, 128, 300])
-@pytest.mark.parametrize("n_q,n_kv,K", [(512, 128, 512), (5120, 1024, 5120), (320, 72, 264)])
+@pytest.mark.parametrize("M", [1, 3, 5, 64, 128, 300, 1000])
+@pytest.mark.parametrize("n_q,n_kv,K", [(512, 128, 512), (5120, 1024, 5120), (320, 72, 264), (352, 96, 520)])
 def test_linear_qkv_writes_the_three_projections(M, n_q, n_kv, K):
     """The fused Q/K/V projection (stacked weight, three output buffers) through its three routes - the streaming
-    kernel (1-4 rows), the cluster split-K kernel (5-128 rows: segment boundaries inside a tile at the odd shape), three
-    large GEMMs (300 rows) - against the oracle's linear per projection; bytes around the outputs stay untouched."""
+    kernel (1-4 rows), the cluster split-K kernel (5-128 rows: segment boundaries inside a tile at the odd shape), one
+    large GEMM whose epilogue writes the three buffers (300 rows: the single-block kernel, 1000 rows: SM pairs; widths
+    that are multiples of 32, also with boundaries inside a 256-column tile) or three large GEMMs (other widths) -
+    against the oracle's linear per projection; bytes around the outputs stay untouched."""
     x = rnd(M, K, seed=11)
     wq, wk, wv = rnd(n_q, K, scale=K ** -0.5, seed=12), rnd(n_kv, K, scale=K ** -0.5, seed=13), rnd(n_kv, K, scale=K ** -0.5, seed=14)
     w_qkv = B().stack_qkv(wq, wk, wv)
