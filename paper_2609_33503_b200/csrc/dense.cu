@@ -450,6 +450,47 @@ carry_rows_kernel(ReqTable rt, const uint16_t* __restrict__ h_in, uint16_t* __re
     *reinterpret_cast<uint4*>(h_out + dst_row * C + i) = __ldg(reinterpret_cast<const uint4*>(h_in + src_row * C + i));
 }
 
+// The same for many rows: one warp per row, the row travels through shared memory by bulk copies (see above).
+__global__ void __launch_bounds__(kRowWarps * 32)
+carry_rows_bulk_kernel(ReqTable rt, const uint16_t* __restrict__ h_in, uint16_t* __restrict__ h_out, int C,
+                       const int* __restrict__ r_rank, const int* __restrict__ r_cu_l, const int* __restrict__ r_cu_next,
+                       DeviceStatus* st) {
+  extern __shared__ __align__(128) uint8_t row_stage[];      // [warp][C] bf16
+  __shared__ __align__(8) unsigned long long bars[kRowWarps];
+  __shared__ volatile int gave_up[kRowWarps];
+  const int B = rt.n_req;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long y = (long long)blockIdx.x * kRowWarps + warp;
+  if (y >= rt.tile_cu[B] || lane != 0) return;                // one lane per row does everything: search, load, store
+  const int b = find_segment(rt.tile_cu, B, (int)y);
+  const int rho = (int)y - rt.tile_cu[b];
+  const int n_next = r_cu_next[b + 1] - r_cu_next[b];
+  if (rho >= n_next) return;
+  const int c = r_rank[r_cu_next[b] + rho];
+  const int* list = r_rank + r_cu_l[b];
+  const int n_l = r_cu_l[b + 1] - r_cu_l[b];
+  int lo = 0, hi = n_l;
+  while (lo < hi) { const int mid = (lo + hi) >> 1; if (list[mid] < c) lo = mid + 1; else hi = mid; }
+  if (lo >= n_l || list[lo] != c) { report(st, RELAXKV_ERR_BAD_INDEX, KID_DENSE, c, lo); return; }
+  const long long src_row = (long long)(r_cu_l[b] - r_cu_l[0]) + lo;
+  const long long dst_row = (long long)(r_cu_next[b] - r_cu_next[0]) + rho;
+  const uint32_t row_bytes = (uint32_t)C * 2;
+  const uint32_t bar = smem_u32(&bars[warp]), stage = smem_u32(row_stage + (size_t)warp * row_bytes);
+  gave_up[warp] = 0;
+  mbar_init(bar, 1);
+  fence_barrier_init();
+  mbar_expect_tx(bar, row_bytes);
+  bulk_load(stage, h_in + src_row * C, row_bytes, bar);
+  if (!mbar_wait(bar, 0, &gave_up[warp])) {
+    report(st, RELAXKV_ERR_TIMEOUT, KID_DENSE, (int)y, -1);
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    return;
+  }
+  bulk_store(h_out + dst_row * C, stage, row_bytes);
+  bulk_store_commit_and_drain();
+}
+
 }  // namespace relaxkv
 
 using namespace relaxkv;
@@ -590,6 +631,15 @@ extern "C" relaxkv_status relaxkv_carry_rows(const relaxkv_shape* shape, const v
   if (total > 0x7fffffffLL) return RELAXKV_ERR_UNSUPPORTED_SHAPE;
   DeviceStatus* st = status_word();
   if (!st) return RELAXKV_ERR_CUDA;
+  if (total >= kRowBulkMinRows && n_cols * 2 <= kRowBulkMaxBytes) {
+    const size_t smem = (size_t)kRowWarps * n_cols * 2;
+    if (smem > 48 * 1024 - 256 &&
+        cudaFuncSetAttribute(carry_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return RELAXKV_ERR_CUDA;
+    carry_rows_bulk_kernel<<<(unsigned)((total + kRowWarps - 1) / kRowWarps), kRowWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+        rt, static_cast<const uint16_t*>(h_in), static_cast<uint16_t*>(h_out), n_cols, r_rank, r_cu_layer, r_cu_next, st);
+    return launch_ok();
+  }
   carry_rows_kernel<<<(unsigned)total, 128, 0, static_cast<cudaStream_t>(stream)>>>(
       rt, static_cast<const uint16_t*>(h_in), static_cast<uint16_t*>(h_out), n_cols, r_rank, r_cu_layer, r_cu_next, st);
   return launch_ok();

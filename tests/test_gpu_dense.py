@@ -198,14 +198,18 @@ def test_qk_norm_rope_in_one_launch(D, with_norm, n, H, Hkv):
     assert torch.equal(qb[0], q0[0]) and torch.equal(qb[n + 1], q0[n + 1]) and torch.equal(kb[0], k0[0]) and torch.equal(kb[n + 1], k0[n + 1])
 
 
-def test_target_positions_and_row_carry():
+@pytest.mark.parametrize("ctx,chunk,C", [((640, 900), 128, 72), ((7000, 9500), 512, 1024)], ids=["few_rows", "many_rows"])
+def test_target_positions_and_row_carry(ctx, chunk, C):
+    """Positions of the targets and the carry of the rows that stay active, bit for bit; with some thousand rows the
+    carry moves whole rows through shared memory by bulk copies."""
     from tests.harness import Case
-    w = inputs.scaled_down(inputs.qwen14b_32k("calibrated"), (640, 900), (9, 17), n_layers=3, chunk=128)
+    w = inputs.scaled_down(inputs.qwen14b_32k("calibrated"), ctx, (9, 17), n_layers=3, chunk=chunk)
     case = Case(w)
     s = case.make_session()
     s.build_active_sets(case.anchors_tensor())
     n_u, n_r = s.counts()
-    C = 72
+    if ctx[0] > 4096:
+        assert sum(n_r[1]) >= 4096                      # the bulk form is the one under test
     for l in range(w.n_layers):
         total = sum(n_r[l])
         pos = torch.full((total,), -1, dtype=torch.int32, device="cuda")
